@@ -1,0 +1,182 @@
+/*
+ * samkv.h — C ABI of the SamKV hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library sparsifies a multiple-context KV cache (per-document K/V that were prefilled
+ * independently of one another) and attends over what survives, following
+ * "Sparse Attention across Multiple-context KV Cache" (SamKV):
+ *
+ *   samkv_score    pooled query, personalised query (Eq. 1), inner-product block scores (Sec. 3.2)
+ *   samkv_select   protected initial/local blocks + per-context top-k of the middle (Sec. 3.2, 4.1)
+ *   samkv_compact  gather of the kept K/V rows into one compact cache, original order (Sec. 3.2)
+ *   samkv_update   write recomputed rows back: Overwrite or Fusion (Sec. 3.3, Eq. 4)
+ *   samkv_attn     GQA attention of a prefill chunk / decode step over the compact cache (Sec. 3.3)
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, innermost dimension
+ *     contiguous, base address 16-byte aligned, unless the comment says "host".
+ *     Arrays marked "host" are read during the call and may be freed right after it returns.
+ *   - Calls validate their arguments on the host, then only enqueue kernels on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream).  They do not allocate,
+ *     free or synchronise (samkv_poll_status is the one call that synchronises).
+ *   - A handle owns no memory: scratch lives in the caller's `workspace`.  Calls that use the
+ *     same handle must be ordered on one stream (they share the workspace).
+ *   - On a host-detected error a call returns a non-zero status and launches nothing.
+ *     Nothing traps or aborts.  There is no CPU fallback.
+ *   - Shapes: L layers, Bt batch elements (independent requests that share the context
+ *     lengths), Hq query heads, Hkv KV heads (Hq % Hkv == 0, G = Hq/Hkv), d = head_dim in {64,128},
+ *     D contexts with ctx_offsets[c] .. ctx_offsets[c+1] on the concatenated token axis of
+ *     length L_tot, B = block_size (selection unit, power of two <= 64; 1 = single tokens),
+ *     units are counted from each context's own start (the last one may be short),
+ *     nb_c = ceil(L_c / B), U_tot = sum nb_c.
+ *   - Protected units of a context: every unit that overlaps its first n_init or last n_local
+ *     tokens (n_init, n_local multiples of B).  If some L_c is not a multiple of B, n_local
+ *     must be >= B so that the short tail unit is protected and every head keeps the same
+ *     number of tokens.
+ */
+#ifndef SAMKV_H_
+#define SAMKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SAMKV_MAX_CTX 128        /* most contexts per request */
+#define SAMKV_MAX_UNITS_PER_CTX 49152  /* most selection units in one context */
+
+typedef struct samkv_ctx* samkv_handle_t; /* opaque */
+
+typedef enum {
+  SAMKV_OK = 0,
+  SAMKV_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, inconsistent sizes */
+  SAMKV_ERR_UNSUPPORTED = 2,  /* head_dim, dtype, block_size or size outside what is built */
+  SAMKV_ERR_WORKSPACE = 3,    /* workspace smaller than samkv_workspace_bytes() */
+  SAMKV_ERR_CAPACITY = 4,     /* compact cache capacity too small */
+  SAMKV_ERR_BUDGET = 5,       /* k_units[c] outside [protected units, nb_c] */
+  SAMKV_ERR_CUDA = 6,         /* a CUDA runtime call failed (launch error, wrong device) */
+  SAMKV_ERR_DEVICE_CHECK = 7  /* a kernel recorded a failed device-side check */
+} samkv_status_t;
+
+typedef enum { SAMKV_F32 = 0, SAMKV_BF16 = 1 } samkv_dtype_t;
+typedef enum { SAMKV_UPDATE_OVERWRITE = 0, SAMKV_UPDATE_FUSION = 1 } samkv_update_mode_t;
+
+/* Problem shape shared by all calls. */
+typedef struct {
+  int32_t n_layers, batch, n_q_heads, n_kv_heads, head_dim;
+  int32_t n_ctx;               /* D, 1 .. SAMKV_MAX_CTX */
+  const int32_t* ctx_offsets;  /* host [n_ctx+1], ascending, ctx_offsets[0] == 0 */
+  int32_t block_size;          /* B; the paper runs with 64 */
+  int32_t n_init, n_local;     /* protected tokens per context; the paper runs with 64 and 128 */
+  int32_t dtype;               /* samkv_dtype_t of K, V, Q, Qloc, Knew, Vnew, Kc, Vc, O */
+} samkv_shape_t;
+
+/* ---- handle, workspace, status -------------------------------------------------------- */
+
+/* Bytes of device scratch the calls below need for this shape: the personalised query
+ * vectors of samkv_score and the split-KV partial results of samkv_attn with up to
+ * max_q_tokens query tokens over a cache of cache_capacity slots.  Returns 0 on a bad shape. */
+size_t samkv_workspace_bytes(const samkv_shape_t* shape, int32_t max_q_tokens, int32_t cache_capacity);
+
+/* Creates a handle bound to CUDA device `device` and to `workspace` (device pointer, 256-byte
+ * aligned, workspace_bytes long, caller-owned, must outlive the handle).  Queries device
+ * properties and enqueues one small memset on the default stream; allocates no device memory. */
+samkv_status_t samkv_create(samkv_handle_t* out, int device, void* workspace, size_t workspace_bytes);
+samkv_status_t samkv_destroy(samkv_handle_t h);
+
+/* Synchronises `stream`, then returns SAMKV_ERR_DEVICE_CHECK if any kernel since the last poll
+ * recorded a failed device-side check (and clears the record), SAMKV_ERR_CUDA if the stream
+ * reports an error, else SAMKV_OK. */
+samkv_status_t samkv_poll_status(samkv_handle_t h, void* stream);
+const char* samkv_status_string(samkv_status_t s);
+
+/* ---- host-side helpers (no GPU work) --------------------------------------------------- */
+
+/* Units kept per context under a sequence budget given in basis points (1500 = 15 %, the
+ * sequence ratio the paper reports in Table 1): k_c = clamp(floor(budget_bp * nb_c / 10000),
+ * protected units of c, nb_c).  k_units_out: host [n_ctx]. */
+samkv_status_t samkv_budget_units(const samkv_shape_t* shape, int32_t budget_bp, int32_t* k_units_out);
+
+/* Number of protected units per context (host [n_ctx], may be NULL) and, for a given k_units
+ * (host [n_ctx], may be NULL), the number of tokens S the compact cache will hold. */
+samkv_status_t samkv_layout(const samkv_shape_t* shape, const int32_t* k_units, int32_t* n_protected_out,
+                            int32_t* total_units_out, int32_t* kept_tokens_out);
+
+/* ---- the five steps --------------------------------------------------------------------- */
+
+/* Scoring (Sec. 3.1 mean pooling; Eq. 1; Sec. 3.2 inner products with block-mean keys).
+ *   K     [L, Bt, Hkv, L_tot, d]
+ *   Q     [L, Bt, T_q, Hq, d]          the user query's Q rows of each layer
+ *   Qloc  [L, Bt, D, T_loc, Hq, d]     each document's local-position Q cache (T_loc = 1 accepts a
+ *                                      pre-pooled vector); NULL or use_bias == 0 => Q^ = Q_que
+ * Per (layer, batch, query head): Q_que = mean_t Q, q_loc_j = mean_t Qloc_j,
+ *   Q^_i = Q_que + 1/(D-1) * sum_{j != i} |cos(Q_que, q_loc_j)| * q_loc_j   (weight 0 for a zero norm;
+ *   D == 1 => Q^ = Q_que), folded to KV heads by the mean over the G query heads of a group.
+ * Per (layer, batch, KV head, token t of context i): s = <q_i, K_t> in fp32 (no scaling);
+ * unit score = mean of s over the unit's real tokens (== <q_i, mean K> by linearity).
+ *   scores_out fp32 [L, Bt, Hkv, U_tot]
+ *   qhat_out   fp32 [L, Bt, D, Hkv, d], optional (NULL: kept in the workspace only) */
+samkv_status_t samkv_score(samkv_handle_t h, const samkv_shape_t* shape, const void* K, const void* Q, int32_t T_q,
+                           const void* Qloc, int32_t T_loc, int32_t use_bias, float* scores_out, float* qhat_out,
+                           void* stream);
+
+/* Selection (Sec. 3.2: initial and local positions are kept in full, the middle is sparsified;
+ * here under a fixed per-context budget).  Per (layer, batch, KV head, context c): keep the
+ * protected units plus the k_units[c] - n_protected_c middle units with the largest score;
+ * of equal scores the lower index wins (-0 and +0 compare equal).
+ *   scores   fp32 [L, Bt, Hkv, U_tot]
+ *   k_units  host [n_ctx], units kept per context, protected ones included
+ *   sel_out  int32 [L, Bt, Hkv, S_u], S_u = sum k_units: global unit ids, ascending;
+ *            context c's segment starts at sum_{c'<c} k_units[c'] */
+samkv_status_t samkv_select(samkv_handle_t h, const samkv_shape_t* shape, const float* scores, const int32_t* k_units,
+                            int32_t* sel_out, void* stream);
+
+/* Compaction (Sec. 3.2: initial + selected + local rows joined in their original order).
+ *   Kc[l,b,h,slot,:] = K[l,b,h,tok(slot),:], same for V; slots run over (context, token) ascending.
+ *   K, V      [L, Bt, Hkv, L_tot, d]
+ *   sel       int32 [L, Bt, Hkv, S_u] as written by samkv_select; k_units host [n_ctx]
+ *   Kc, Vc    [L, Bt, Hkv, cache_capacity, d]; slots >= S are left untouched
+ *   cache_len int32 [L, Bt], set to S (the number of kept tokens)
+ *   inv_map   int32 [L, Bt, Hkv, L_tot], optional: slot of each token, -1 where this head did not
+ *             keep it (the paper's "blank" position when layers/heads are aligned for recomputation)
+ * Returns SAMKV_ERR_CAPACITY if cache_capacity < S.  Copies are bit-exact. */
+samkv_status_t samkv_compact(samkv_handle_t h, const samkv_shape_t* shape, const void* K, const void* V,
+                             const int32_t* sel, const int32_t* k_units, void* Kc, void* Vc, int32_t cache_capacity,
+                             int32_t* cache_len, int32_t* inv_map, void* stream);
+
+/* Write-back of recomputed rows (Sec. 3.3).  For every recomputed token r and every KV head that
+ * kept it (slot = inv_map[l,b,h,tok_ids[l,r]] >= 0):
+ *   overwrite: Kc[slot] = Knew[r], Vc[slot] = Vnew[r]
+ *   fusion (Eq. 4): theta = cos(new, old) over the d elements of the row (1 if a norm is zero),
+ *                   row = theta*new + (1-theta)*old in fp32, rounded to nearest-even in dtype;
+ *                   K rows and V rows each use their own theta.
+ *   tok_ids    int32 [L, R] global token ids on the concatenated axis, -1 = skip; ids of one layer
+ *              must be distinct
+ *   Knew, Vnew [L, Bt, R, Hkv, d] */
+samkv_status_t samkv_update(samkv_handle_t h, const samkv_shape_t* shape, void* Kc, void* Vc, int32_t cache_capacity,
+                            const int32_t* inv_map, const int32_t* tok_ids, int32_t R, const void* Knew,
+                            const void* Vnew, int32_t mode, void* stream);
+
+/* Attention of a query chunk over the compact cache of one layer (Sec. 3.3: the incremental
+ * prefill of the user query over the new sparse cache, and the decode steps after it).
+ *   Kc, Vc    [L, Bt, Hkv, cache_capacity, d]; `layer` picks the slab
+ *   cache_len int32 [L, Bt] (device).  Slots < cache_len[layer,b] are visible to every query token.
+ *   Q         [Bt, T_q, Hq, d] fresh query rows of this step
+ *   Kq, Vq    [Bt, T_q, Hkv, d] optional (both or neither): the chunk's own keys/values, written to
+ *             slots cache_len .. cache_len+T_q-1 and attended causally (token t sees appended slots <= t);
+ *             afterwards cache_len[layer,b] += T_q.  The caller guarantees cache_len + T_q <= cache_capacity
+ *             (a violation is recorded as a device check and the append is skipped).
+ *   scale     softmax scale; <= 0 selects 1/sqrt(d)
+ *   O         [Bt, T_q, Hq, d] = softmax(scale * Q Kc^T + mask) Vc, query head hq reads KV head hq/G
+ *   lse       fp32 [Bt, Hq, T_q] optional: log of the softmax denominator
+ * bf16 inputs: products on tensor cores with fp32 accumulation, probabilities rounded to bf16
+ * before the PV product.  fp32 inputs: fp32 FMA throughout. */
+samkv_status_t samkv_attn(samkv_handle_t h, const samkv_shape_t* shape, int32_t layer, void* Kc, void* Vc,
+                          int32_t cache_capacity, int32_t* cache_len, const void* Q, int32_t T_q, const void* Kq,
+                          const void* Vq, float scale, void* O, float* lse, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAMKV_H_ */

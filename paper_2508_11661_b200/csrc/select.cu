@@ -1,0 +1,144 @@
+// Per-context selection of SamKV (Sec. 3.2): protected initial/local units are always kept, the
+// middle units compete under a fixed budget.  One CTA per (layer, batch, kv head, context):
+// the middle scores are turned into order-preserving 32-bit keys held in shared memory, an
+// MSB-first radix select (4 passes of 8 bits) finds the k-th largest key, ties at that key are
+// broken by index order with a block scan, and the kept ids are emitted already ascending.
+#include "common.cuh"
+
+namespace samkv {
+
+constexpr int kSelThreads = 256;
+
+// float -> uint32 with the same ordering; -0 and +0 map to the same key.
+__device__ __forceinline__ uint32_t score_key(float x) {
+  uint32_t u = __float_as_uint(x);
+  if ((u << 1) == 0) u = 0;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive prefix sum over the kSelThreads values held one per thread; also returns the total.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  __syncthreads();
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  uint32_t before = 0, tot = 0;
+#pragma unroll
+  for (int i = 0; i < kSelThreads / 32; ++i) {
+    const uint32_t t = warp_tot[i];
+    if (i < warp) before += t;
+    tot += t;
+  }
+  *total = tot;
+  return before + inc - v;
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const float* __restrict__ scores, int32_t* __restrict__ sel, const __grid_constant__ CtxTable ct,
+              const __grid_constant__ SelTable st, int U_tot, int S_u, int* __restrict__ d_status) {
+  extern __shared__ uint32_t keys[];         // [n_mid]
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t warp_tot[kSelThreads / 32];
+  __shared__ uint32_t s_bin, s_remaining;
+
+  const int c = blockIdx.x % ct.n_ctx;
+  const size_t slab = blockIdx.x / ct.n_ctx;
+  const int base = ct.unit_off[c];
+  const int nb = ct.unit_off[c + 1] - base;
+  const int p0 = st.n_init_units[c];          // middle units are [p0, p1)
+  const int p1 = st.first_local_unit[c];
+  const int k = st.sel_off[c + 1] - st.sel_off[c];
+  const int n_mid = p1 - p0;
+  const int k_mid = k - (nb - n_mid);
+  int32_t* out = sel + slab * S_u + st.sel_off[c];
+  const int tid = threadIdx.x;
+
+  for (int i = tid; i < p0; i += kSelThreads) out[i] = base + i;
+  for (int i = p1 + tid; i < nb; i += kSelThreads) out[k - (nb - p1) + (i - p1)] = base + i;
+  if (k_mid <= 0) return;
+  if (k_mid >= n_mid) {
+    for (int i = tid; i < n_mid; i += kSelThreads) out[p0 + i] = base + p0 + i;
+    return;
+  }
+
+  const float* sc = scores + slab * U_tot + base + p0;
+  for (int i = tid; i < n_mid; i += kSelThreads) keys[i] = score_key(sc[i]);
+
+  // ---- radix select: the k_mid-th largest key ----
+  uint32_t prefix = 0, mask = 0, remaining = (uint32_t)k_mid;
+#pragma unroll 1
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    hist[tid] = 0;
+    __syncthreads();   // also orders the key writes before the first pass
+    for (int i = tid; i < n_mid; i += kSelThreads) {
+      const uint32_t key = keys[i];
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    // count of candidates in bins above `tid`: total - inclusive prefix
+    const uint32_t mine = hist[tid];
+    uint32_t total;
+    const uint32_t below = block_exclusive_scan(mine, warp_tot, &total);
+    const uint32_t above = total - below - mine;
+    if (above < remaining && above + mine >= remaining) {   // exactly one bin satisfies this
+      s_bin = tid;
+      s_remaining = remaining - above;
+    }
+    __syncthreads();
+    prefix |= s_bin << shift;
+    mask |= 255u << shift;
+    remaining = s_remaining;
+    __syncthreads();
+  }
+  const uint32_t pivot = prefix;       // k-th largest key
+  const uint32_t need_eq = remaining;  // how many keys equal to the pivot are kept (lowest indices first)
+
+  // ---- ordered compaction: contiguous segment per thread, packed (greater, equal) counts ----
+  const int per = (n_mid + kSelThreads - 1) / kSelThreads;
+  const int a = min(tid * per, n_mid), b = min(a + per, n_mid);
+  uint32_t gt = 0, eq = 0;
+  for (int i = a; i < b; ++i) {
+    const uint32_t key = keys[i];
+    gt += key > pivot;
+    eq += key == pivot;
+  }
+  uint32_t total;
+  const uint32_t packed = block_exclusive_scan((gt << 16) | eq, warp_tot, &total);
+  uint32_t gt_before = packed >> 16, eq_before = packed & 0xffffu;
+  for (int i = a; i < b; ++i) {
+    const uint32_t key = keys[i];
+    if (key > pivot) {
+      out[p0 + gt_before + min(eq_before, need_eq)] = base + p0 + i;
+      ++gt_before;
+    } else if (key == pivot) {
+      if (eq_before < need_eq) out[p0 + gt_before + eq_before] = base + p0 + i;
+      ++eq_before;
+    }
+  }
+  (void)d_status;
+}
+
+cudaError_t launch_select(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const float* scores,
+                          const int32_t* k_units_host, int max_units, int32_t* sel, int* d_status,
+                          cudaStream_t stream) {
+  (void)k_units_host;
+  const long long blocks = (long long)s.n_layers * s.batch * s.n_kv_heads * ct.n_ctx;
+  if (blocks == 0) return cudaSuccess;
+  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+  const size_t smem = (size_t)max_units * sizeof(uint32_t);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  select_kernel<<<(unsigned)blocks, kSelThreads, smem, stream>>>(scores, sel, ct, st, ct.unit_off[ct.n_ctx],
+                                                                st.sel_off[ct.n_ctx], d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace samkv

@@ -1,0 +1,255 @@
+"""GPU-vs-oracle parity, stage by stage, through the C ABI (libsamkv.so via the ctypes binding).
+
+Acceptance (stated in samkv_testlib): selected index sets exact except inside the 1e-5 relative
+tie band around the oracle's k-th score; compaction bit-exact; overwrite bit-exact; fusion within
+one bf16 ulp (bf16) / 1e-5 relative (fp32); attention max-abs <= 2e-2 (bf16) / 1e-4 (fp32).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import samkv_oracle as O
+from paper_2508_11661_b200 import binding as B
+from paper_2508_11661_b200 import synth
+from samkv_testlib import (GpuRun, check_attention, check_compact, check_scores, check_selection, check_update,
+                           oracle_k_units, oracle_scores, to_f64)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def full_check(w, inp=None, k_units=None, use_bias=True, with_qloc=True, append=True, layers=None, batches=None):
+    """Sparsify + prefill attention for a workload; every stage against the oracle."""
+    inp = inp if inp is not None else {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp, k_units=k_units, use_bias=use_bias, with_qloc=with_qloc).sparsify()
+    if k_units is None:
+        assert run.k_units == oracle_k_units(w)
+    torch.cuda.synchronize()
+    sel = run.sel.cpu().numpy()
+    n_diff = 0
+    ls = list(layers if layers is not None else range(w.n_layers))
+    bs = list(batches if batches is not None else range(w.batch))
+    for l in ls:
+        for b in bs:
+            q, s, u = oracle_scores(w, inp, l, b, use_bias, with_qloc)
+            check_scores(w, run, l, b, q, u)
+            n_diff += check_selection(w, run.k_units, sel[l, b], u, where=f"{w.name} l{l} b{b}")
+            check_compact(w, run, l, b, sel[l, b])
+    for l in ls:
+        Kc_before, Vc_before = run.Kc[l].clone(), run.Vc[l].clone()
+        Kq = inp["Kq"][l] if append else None
+        Vq = inp["Vq"][l] if append else None
+        Og, lse = run.attn(l, inp["Qa"][l], Kq, Vq)
+        torch.cuda.synchronize()
+        for b in bs:
+            err, K2, V2, n = check_attention(w, Kc_before[b], Vc_before[b], run.S, inp["Qa"][l, b],
+                                             Kq[b] if append else None, Vq[b] if append else None, Og[b], lse[b])
+            assert int(run.cache_len[l, b]) == n
+            if append:    # appended rows are in the cache, bit-exact, right after the kept tokens
+                assert np.array_equal(to_f64(run.Kc[l, b][:, run.S:n]), K2[:, run.S:n])
+                assert np.array_equal(to_f64(run.Vc[l, b][:, run.S:n]), V2[:, run.S:n])
+    assert run.poll() == 0
+    return run, n_diff
+
+
+def test_cfg0_tiny_fp32():
+    run, _ = full_check(synth.CONFIGS["cfg0"])
+    assert run.S == 152
+
+
+def test_cfg1_llama_shape_bf16():
+    run, _ = full_check(synth.CONFIGS["cfg1"])
+    assert run.S == 1530
+
+
+@pytest.mark.parametrize("dtype,hd", [("f32", 64), ("f32", 128), ("bf16", 64), ("bf16", 128)])
+def test_ragged_contexts_token_mode(dtype, hd):
+    w = synth.ragged_workload(dtype=dtype, head_dim=hd, n_q_heads=6, n_kv_heads=2, q_tokens=5)
+    full_check(w)
+
+
+@pytest.mark.parametrize("B_,ni,nl", [(16, 16, 32), (64, 64, 128), (4, 4, 8), (2, 0, 2)])
+def test_block_mode_ragged(B_, ni, nl):
+    w = synth.ragged_workload(ctx_lens=(300, 1027, 256, 2000), dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=2,
+                              q_tokens=9, block_size=B_, n_init=ni, n_local=nl, budget_bp=2000)
+    full_check(w)
+
+
+def test_block_mode_cfg1_paper_blocks():
+    full_check(synth.CONFIGS["cfg1"].replace(name="cfg1_b64", block_size=64, n_init=64, n_local=128, budget_bp=3000))
+    full_check(synth.CONFIGS["cfg0"].replace(name="cfg0_b16", block_size=16, n_init=16, n_local=32, budget_bp=4000))
+
+
+def test_single_context_and_bias_switches():
+    w = synth.ragged_workload(ctx_lens=(700,), dtype="bf16", head_dim=128, n_q_heads=8, n_kv_heads=4, q_tokens=3)
+    run, _ = full_check(w)                                        # D = 1: Q^ = Q_que
+    w4 = synth.ragged_workload(dtype="f32", head_dim=64)
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w4, "cpu").items()}
+    a, _ = full_check(w4, inp, use_bias=False)
+    b, _ = full_check(w4, inp, with_qloc=False)
+    assert torch.equal(a.scores, b.scores) and torch.equal(a.sel, b.sel)
+    c, _ = full_check(w4, inp, use_bias=True)
+    assert not torch.equal(a.scores, c.scores)
+
+
+def test_budget_edges_protected_only_and_full():
+    w = synth.ragged_workload(dtype="bf16", head_dim=128, n_q_heads=4, n_kv_heads=2)
+    shape = B.Shape.from_workload(w)
+    prot, _, _ = B.samkv_layout(shape)
+    run, _ = full_check(w, k_units=prot)                          # the "no selection" ablation: protected only
+    assert run.S == sum(prot)
+    nb = list(w.ctx_lens)
+    run, _ = full_check(w, k_units=nb, append=False)              # 100 %
+    assert run.S == w.l_tot
+    # 100 % budget, no update: identical to full attention over the concatenated contexts
+    inp = run.inp
+    assert torch.equal(run.Kc[0, 0][:, :w.l_tot], inp["K"][0, 0]) and torch.equal(run.Vc[0, 0][:, :w.l_tot], inp["V"][0, 0])
+    Og, _ = run.attn(0, inp["Qa"][0])
+    out, *_ = O.attention(to_f64(inp["K"][0, 0]), to_f64(inp["V"][0, 0]), w.l_tot, to_f64(inp["Qa"][0, 0]))
+    assert np.abs(to_f64(Og[0]) - out).max() <= 2e-2
+
+
+def test_ties_lower_index_wins():
+    """Duplicated key rows give exactly equal scores on both sides; the lower index must be kept."""
+    w = synth.ragged_workload(ctx_lens=(400, 600), dtype="bf16", head_dim=128, n_q_heads=4, n_kv_heads=2, n_init=4,
+                              n_local=4, budget_bp=1000)
+    inp = synth.make_inputs(w, "cpu")
+    K = inp["K"]
+    g = torch.Generator().manual_seed(5)
+    for h in range(2):
+        for c, (lo, hi) in enumerate(((0, 400), (400, 1000))):
+            src = torch.randint(lo + 10, hi - 10, (60,), generator=g)
+            dst = torch.randint(lo + 10, hi - 10, (60,), generator=g)
+            K[0, 0, h, dst] = K[0, 0, h, src]
+    # and a context where every middle key is the same row: the kept middle units must be the first ones
+    K[0, 0, 0, 404:996] = K[0, 0, 0, 500]
+    inp = {k: v.to(DEV) for k, v in inp.items()}
+    run, n_diff = full_check(w, inp)
+    sel = run.sel[0, 0, 0].cpu().numpy()
+    k0, k1 = run.k_units
+    mid = sel[k0 + 4: k0 + k1 - 4]
+    assert list(mid) == list(range(404, 404 + len(mid)))
+
+
+@pytest.mark.parametrize("mode", [B.SAMKV_UPDATE_OVERWRITE, B.SAMKV_UPDATE_FUSION])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_update_overwrite_and_fusion(mode, dtype):
+    """Reduced cfg2: outlier channels, sink keys, 15 % of the kept tokens recomputed, then attention."""
+    w = synth.CONFIGS["cfg2"].replace(name="cfg2_small", n_layers=2, batch=2, ctx_lens=(384, 256, 512), dtype=dtype,
+                                      q_tokens=16)
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp).sparsify()
+    sel = run.sel.cpu().numpy()
+    toks0 = np.stack([[O.units_to_tokens(sel[l, b, 0], w.ctx_offsets, 1) for b in range(w.batch)]
+                      for l in range(w.n_layers)])
+    R = (w.recompute_share_bp * run.S) // 10000
+    tok_ids, Knew, Vnew = synth.make_recompute(w, inp["K"], inp["V"], torch.from_numpy(toks0), R)
+    tok_ids[0, 3] = -1                                             # a skipped entry
+    Kc0, Vc0 = run.Kc.clone(), run.Vc.clone()
+    run.update(tok_ids, Knew, Vnew, mode)
+    torch.cuda.synchronize()
+    inv = run.inv_map.cpu().numpy()
+    n_blank = 0
+    for l in range(w.n_layers):
+        for b in range(w.batch):
+            check_update(w, Kc0[l, b], Vc0[l, b], run.Kc[l, b], run.Vc[l, b], inv[l, b], tok_ids[l].cpu().numpy(),
+                         Knew[l, b], Vnew[l, b], mode)
+            n_blank += int((inv[l, b][1:, tok_ids[l].cpu().numpy().clip(0)] < 0).sum())
+        Og, lse = run.attn(l, inp["Qa"][l], inp["Kq"][l], inp["Vq"][l])
+        for b in range(w.batch):
+            check_attention(w, run.Kc[l, b].clone(), run.Vc[l, b].clone(), run.S, inp["Qa"][l, b], inp["Kq"][l, b],
+                            inp["Vq"][l, b], Og[b], lse[b])
+    assert n_blank > 0          # some heads did not keep some recomputed tokens: the skip rule was exercised
+    assert run.poll() == 0
+
+
+def test_decode_steps_append_to_compact_cache():
+    """Reduced cfg3: sparsify, prefill a 32-token chunk, then decode steps of one token each."""
+    w = synth.CONFIGS["cfg3"].replace(name="cfg3_small", batch=3, ctx_lens=(512, 768, 300), decode_steps=12)
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp).sparsify()
+    Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+    Kc_ref = [to_f64(run.Kc[0, b]) for b in range(w.batch)]
+    Vc_ref = [to_f64(run.Vc[0, b]) for b in range(w.batch)]
+    n = run.S + w.q_tokens
+    g = torch.Generator().manual_seed(9)
+    for step in range(w.decode_steps):
+        q = torch.randn((w.batch, 1, w.n_q_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        kq = torch.randn((w.batch, 1, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        vq = torch.randn((w.batch, 1, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        Os, ls = run.attn(0, q, kq, vq)
+        for b in range(w.batch):
+            out, l2, Kc_ref[b], Vc_ref[b], n2 = O.attention(Kc_ref[b], Vc_ref[b], n, to_f64(q[b]), to_f64(kq[b]), to_f64(vq[b]))
+            assert np.abs(to_f64(Os[b]) - out).max() <= 2e-2
+            assert np.abs(to_f64(ls[b]) - l2).max() <= 2e-2
+        n += 1
+        assert run.cache_len.cpu().tolist() == [[n] * w.batch]
+    for b in range(w.batch):
+        assert np.array_equal(to_f64(run.Kc[0, b])[:, :n], Kc_ref[b][:, :n])
+    assert run.poll() == 0
+
+
+@pytest.mark.parametrize("T_q,G", [(1, 4), (8, 4), (3, 8), (40, 4), (64, 8)])
+def test_attention_row_tilings_and_long_cache(T_q, G):
+    """Every row tiling of the bf16 kernel (16 / 64 / 128 packed rows per CTA), with many KV splits."""
+    w = synth.ragged_workload(ctx_lens=(3000, 2500), dtype="bf16", head_dim=128, n_q_heads=2 * G, n_kv_heads=2,
+                              q_tokens=T_q, n_init=16, n_local=32, budget_bp=9000)
+    full_check(w)
+
+
+def test_results_are_deterministic():
+    w = synth.CONFIGS["cfg1"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    outs = []
+    for _ in range(3):
+        run = GpuRun(w, inp).sparsify()
+        Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+        outs.append((run.scores.clone(), run.sel.clone(), run.Kc.clone(), Og.clone(), lse.clone()))
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+
+
+def test_error_codes_launch_nothing():
+    w = synth.CONFIGS["cfg0"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    sel_before = run.sel.clone()
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_select(run.handle, run.shape, run.scores, [5, 38, 38, 38], run.sel)         # below the protected count
+    assert e.value.status == 5
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_select(run.handle, run.shape, run.scores, [257, 38, 38, 38], run.sel)
+    assert e.value.status == 5
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_compact(run.handle, run.shape, inp["K"], inp["V"], run.sel, run.k_units, run.Kc, run.Vc, 100,
+                        run.cache_len, None)
+    assert e.value.status == 4
+    with pytest.raises(B.SamkvError) as e:                                                   # misaligned K
+        B.samkv_score(run.handle, run.shape, inp["K"].view(-1)[1:], inp["Q"], 16, None, 1, 0, run.scores, None)
+    assert e.value.status == 1
+    bad = B.Shape(1, 1, 4, 2, 96, w.ctx_offsets, 1, 4, 8, "f32")
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_score(run.handle, bad, inp["K"], inp["Q"], 16, None, 1, 0, run.scores, None)
+    assert e.value.status == 2
+    with pytest.raises(B.SamkvError) as e:                                                   # Kq without Vq
+        B.samkv_attn(run.handle, run.shape, 0, run.Kc, run.Vc, run.capacity, run.cache_len, inp["Qa"][0], 16,
+                     inp["Kq"][0], None, 0.0, torch.empty_like(inp["Qa"][0]))
+    assert e.value.status == 1
+    torch.cuda.synchronize()
+    assert torch.equal(run.sel, sel_before) and run.poll() == 0
+
+
+def test_append_past_capacity_is_reported_not_fatal():
+    """A full cache: the append is skipped, a device check is recorded, the context stays usable."""
+    w = synth.CONFIGS["cfg0"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp, extra_capacity=8).sparsify()               # room for 8 tokens, chunk has 16
+    Og, _ = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+    assert run.poll() == 7
+    assert int(run.cache_len[0, 0]) == run.S
+    assert run.poll() == 0                                          # cleared by the previous poll
+    Og2, _ = run.attn(0, inp["Qa"][0])                              # cache-only attention still works
+    check_attention(w, run.Kc[0, 0], run.Vc[0, 0], run.S, inp["Qa"][0, 0], None, None, Og2[0])
+    assert torch.equal(Og, Og2)
