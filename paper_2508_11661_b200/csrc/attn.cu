@@ -54,9 +54,10 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
 // ---------------------------------------------------------------------------------------------
 __global__ void append_kernel(char* __restrict__ Kc, char* __restrict__ Vc, const int32_t* __restrict__ cache_len,
                               const char* __restrict__ Kq, const char* __restrict__ Vq, int Hkv, int T_q, int capacity,
-                              int row_bytes, int* __restrict__ d_status) {
+                              int row_bytes, long long n_threads, int* __restrict__ d_status) {
   const int lanes = row_bytes / 16;
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= n_threads) return;
   const long long row = gid / lanes;                // (b * T_q + t) * Hkv + h
   const int lane = (int)(gid % lanes);
   const int h = (int)(row % Hkv);
@@ -243,7 +244,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
     const long long threads = (long long)Bt * T_q * Hkv * (row_bytes / 16);
     append_kernel<<<(unsigned)((threads + 127) / 128), 128, 0, stream>>>((char*)Kl, (char*)Vl, len_l, (const char*)Kq,
                                                                         (const char*)Vq, Hkv, T_q, capacity, row_bytes,
-                                                                        d_status);
+                                                                        threads, d_status);
   }
   const int G = Hq / Hkv;
   const int rows = T_q * G;

@@ -1,0 +1,153 @@
+"""Parity at the benchmark description's full sizes (cfg2, cfg3, cfg4), in the launch configuration
+bench.py times.  Inputs are generated on the GPU (seeded); the oracle reads host copies of sampled
+(layer, batch element) problems, so both sides see the same stored values."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import samkv_oracle as O
+from paper_2508_11661_b200 import binding as B
+from paper_2508_11661_b200 import synth
+from samkv_testlib import (GpuRun, check_attention, check_compact, check_scores, check_selection, check_update,
+                           oracle_scores, to_f64)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _free_all():
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+def test_cfg2_full_size_sampled_slabs():
+    """32 layers x batch 4 x 20 contexts x 1536 tokens, outlier channels + sink keys, 15 % budget,
+    fusion update of 15 % of the kept tokens, attention with the appended 64-token chunk."""
+    w = synth.CONFIGS["cfg2"]
+    inp = synth.make_inputs(w, DEV)
+    run = GpuRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    assert run.S == 4600 and run.poll() == 0
+    samples = [(0, 0), (17, 2), (31, 3)]
+    sel_s = {lb: run.sel[lb].cpu().numpy() for lb in samples}
+    n_diff = 0
+    for (l, b) in samples:
+        q, s, u = oracle_scores(w, inp, l, b)
+        check_scores(w, run, l, b, q, u)
+        n_diff += check_selection(w, run.k_units, sel_s[(l, b)], u, where=f"cfg2 l{l} b{b}")
+        check_compact(w, run, l, b, sel_s[(l, b)])
+    # every slab: ascending ids, per-context counts, protected units present (properties that hold at any size)
+    sel = run.sel
+    assert bool((sel[..., 1:] > sel[..., :-1]).all())
+    nb, off = O.unit_layout(w.ctx_offsets, 1)
+    pos = 0
+    for c in range(w.n_ctx):
+        seg = sel[..., pos:pos + run.k_units[c]]
+        assert bool(((seg >= off[c]) & (seg < off[c + 1])).all())
+        assert bool((seg[..., :w.n_init] == torch.arange(off[c], off[c] + w.n_init, device=DEV, dtype=torch.int32)).all())
+        assert bool((seg[..., -w.n_local:] == torch.arange(off[c + 1] - w.n_local, off[c + 1], device=DEV, dtype=torch.int32)).all())
+        pos += run.k_units[c]
+    # update (fusion) with the benchmark's recompute recipe
+    inv0 = run.inv_map[:, :1, 0, :]
+    toks0 = torch.stack([torch.nonzero(inv0[l, 0] >= 0).flatten() for l in range(w.n_layers)])[:, None, :]
+    R = (w.recompute_share_bp * run.S) // 10000
+    assert R == 690
+    tok_ids, Knew, Vnew = synth.make_recompute(w, inp["K"], inp["V"], toks0, R)
+    before = {lb: (run.Kc[lb].clone(), run.Vc[lb].clone()) for lb in samples}
+    run.update(tok_ids, Knew, Vnew, B.SAMKV_UPDATE_FUSION)
+    torch.cuda.synchronize()
+    for (l, b) in samples:
+        check_update(w, before[(l, b)][0], before[(l, b)][1], run.Kc[l, b], run.Vc[l, b],
+                     run.inv_map[l, b].cpu().numpy(), tok_ids[l].cpu().numpy(), Knew[l, b], Vnew[l, b],
+                     B.SAMKV_UPDATE_FUSION)
+    for l in sorted({l for l, _ in samples}):
+        snap = {b: (run.Kc[l, b].clone(), run.Vc[l, b].clone()) for (ll, b) in samples if ll == l}
+        Og, lse = run.attn(l, inp["Qa"][l], inp["Kq"][l], inp["Vq"][l])
+        torch.cuda.synchronize()
+        for b, (kc, vc) in snap.items():
+            check_attention(w, kc, vc, run.S, inp["Qa"][l, b], inp["Kq"][l, b], inp["Vq"][l, b], Og[b], lse[b])
+    assert run.poll() == 0
+    del run, inp
+    _free_all()
+
+
+def test_cfg3_full_size_decode_128_steps():
+    """batch 32, 10 contexts x 2048 tokens compacted to 15 %, a 32-token prefill chunk, then 128 decode
+    steps of one token each appending to the compact cache; sampled batch elements follow every step."""
+    w = synth.CONFIGS["cfg3"]
+    inp = synth.make_inputs(w, DEV)
+    run = GpuRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    assert run.S == 3070
+    sample_b = [0, 13, 31]
+    sel = run.sel[0].cpu().numpy()
+    for b in sample_b:
+        q, s, u = oracle_scores(w, inp, 0, b)
+        check_selection(w, run.k_units, sel[b], u, where=f"cfg3 b{b}")
+        check_compact(w, run, 0, b, sel[b])
+    snap = {b: (run.Kc[0, b].clone(), run.Vc[0, b].clone()) for b in sample_b}
+    Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+    torch.cuda.synchronize()
+    ref = {}
+    for b in sample_b:
+        _, K2, V2, n = check_attention(w, snap[b][0], snap[b][1], run.S, inp["Qa"][0, b], inp["Kq"][0, b],
+                                       inp["Vq"][0, b], Og[b], lse[b])
+        ref[b] = (K2, V2)
+    n = run.S + w.q_tokens
+    g = torch.Generator(device=DEV).manual_seed(77)
+    shp_q = (w.batch, 1, w.n_q_heads, w.head_dim)
+    shp_k = (w.batch, 1, w.n_kv_heads, w.head_dim)
+    worst = 0.0
+    for step in range(w.decode_steps):
+        q = torch.randn(shp_q, generator=g, device=DEV).to(w.torch_dtype)
+        kq = torch.randn(shp_k, generator=g, device=DEV).to(w.torch_dtype)
+        vq = torch.randn(shp_k, generator=g, device=DEV).to(w.torch_dtype)
+        Os, ls = run.attn(0, q, kq, vq)
+        for b in sample_b:
+            out, l2, K2, V2, n2 = O.attention(ref[b][0], ref[b][1], n, to_f64(q[b]), to_f64(kq[b]), to_f64(vq[b]))
+            ref[b] = (K2, V2)
+            err = np.abs(to_f64(Os[b]) - out).max()
+            worst = max(worst, err)
+            assert err <= 2e-2, f"step {step} b{b}: {err}"
+        n += 1
+    assert run.cache_len.cpu().tolist() == [[n] * w.batch] and n == run.capacity
+    for b in sample_b:
+        assert np.array_equal(to_f64(run.Kc[0, b]), ref[b][0]) and np.array_equal(to_f64(run.Vc[0, b]), ref[b][1])
+    assert run.poll() == 0
+    del run, inp
+    _free_all()
+
+
+@pytest.mark.parametrize("budget_bp", [500, 1500, 3000, 10000])
+def test_cfg4_stress_budget_sweep(budget_bp):
+    """64 query heads / 8 KV heads, 50 contexts x 2048 tokens, 128 query tokens.  At 100 % the result
+    must equal full attention over the concatenated contexts (oracle run on the original K/V)."""
+    w = synth.CONFIGS["cfg4"].replace(budget_bp=budget_bp)
+    inp = synth.make_inputs(w, DEV)
+    run = GpuRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    assert run.S == {500: 5100, 1500: 15350, 3000: 30700, 10000: 102400}[budget_bp]
+    sel = run.sel[0, 0].cpu().numpy()
+    q, s, u = oracle_scores(w, inp, 0, 0)
+    check_scores(w, run, 0, 0, q, u)
+    check_selection(w, run.k_units, sel, u, where=f"cfg4@{budget_bp}")
+    check_compact(w, run, 0, 0, sel)
+    t_sample = [0, 63, 127]
+    Og, lse = run.attn(0, inp["Qa"][0], None, None)                  # cache-only attention
+    torch.cuda.synchronize()
+    if budget_bp == 10000:
+        check_attention(w, inp["K"][0, 0], inp["V"][0, 0], w.l_tot, inp["Qa"][0, 0], None, None, Og[0], lse[0],
+                        t_sample=t_sample)
+    else:
+        check_attention(w, run.Kc[0, 0], run.Vc[0, 0], run.S, inp["Qa"][0, 0], None, None, Og[0], lse[0],
+                        t_sample=t_sample)
+    # and the prefill form with the chunk appended
+    snap = (run.Kc[0, 0].clone(), run.Vc[0, 0].clone()) if budget_bp <= 1500 else None
+    Og2, lse2 = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+    torch.cuda.synchronize()
+    if snap is not None:
+        check_attention(w, snap[0], snap[1], run.S, inp["Qa"][0, 0], inp["Kq"][0, 0], inp["Vq"][0, 0], Og2[0], lse2[0])
+    assert int(run.cache_len[0, 0]) == run.S + w.q_tokens and run.poll() == 0
+    del run, inp
+    _free_all()
