@@ -164,26 +164,34 @@ def bf16_ulp(x: np.ndarray) -> np.ndarray:
 
 
 def check_update(w, Kc_before, Vc_before, Kc_after, Vc_after, inv_lb, tok_ids_l, Knew_lb, Vnew_lb, mode):
-    """Overwrite: bit-exact.  Fusion: fp32 inputs within 1e-5 relative of the row norm; bf16 within one
-    bf16 unit in the last place of the oracle value (the fp32 theta and the fp64 theta can round
-    differently).  Untouched slots must be bit-identical."""
+    """Overwrite: bit-exact.  Fusion: the GPU forms theta and the blend in fp32, the oracle in fp64, and
+    both round the row to the cache dtype, so an element may differ by one unit in the last place of
+    the oracle value, plus the fp32 error of the blend, which scales with the operands (not with a
+    result that may have cancelled): 1e-5 * (|new| + |old|) per element.  fp32 caches: 1e-5 of the row
+    norm.  Untouched slots must be bit-identical."""
     mode_name = "overwrite" if mode == B.SAMKV_UPDATE_OVERWRITE else "fusion"
-    Ko, Vo = O.update(to_f64(Kc_before), to_f64(Vc_before), inv_lb, tok_ids_l, to_f64(Knew_lb), to_f64(Vnew_lb),
-                      mode_name, dtype=w.dtype if w.dtype != "f32" else "f32")
+    Kb, Vb = to_f64(Kc_before), to_f64(Vc_before)
+    Kn, Vn = to_f64(Knew_lb), to_f64(Vnew_lb)
+    Ko, Vo = O.update(Kb, Vb, inv_lb, tok_ids_l, Kn, Vn, mode_name, dtype=w.dtype)
     Kg, Vg = to_f64(Kc_after), to_f64(Vc_after)
     touched = np.zeros(Kg.shape[:2], dtype=bool)
-    for tok in tok_ids_l:
+    mag_k, mag_v = np.zeros_like(Kg), np.zeros_like(Vg)
+    for r, tok in enumerate(tok_ids_l):
         if tok >= 0:
             for h in range(Kg.shape[0]):
-                if inv_lb[h, tok] >= 0:
-                    touched[h, inv_lb[h, tok]] = True
-    assert np.array_equal(Kg[~touched], to_f64(Kc_before)[~touched]) and np.array_equal(Vg[~touched], to_f64(Vc_before)[~touched])
+                slot = inv_lb[h, tok]
+                if slot >= 0:
+                    touched[h, slot] = True
+                    mag_k[h, slot] = np.abs(Kn[r, h]) + np.abs(Kb[h, slot])
+                    mag_v[h, slot] = np.abs(Vn[r, h]) + np.abs(Vb[h, slot])
+    assert np.array_equal(Kg[~touched], Kb[~touched]) and np.array_equal(Vg[~touched], Vb[~touched])
     if mode_name == "overwrite":
         assert np.array_equal(Kg, Ko) and np.array_equal(Vg, Vo)
         return
-    for got, exp in ((Kg, Ko), (Vg, Vo)):
+    for got, exp, mag in ((Kg, Ko, mag_k), (Vg, Vo, mag_v)):
         if w.dtype == "bf16":
-            assert np.all(np.abs(got - exp)[touched] <= bf16_ulp(exp)[touched] + 1e-30)
+            tol = bf16_ulp(exp) + 1e-5 * mag
+            assert np.all(np.abs(got - exp)[touched] <= tol[touched])
         else:
             nrm = np.sqrt((exp ** 2).sum(-1, keepdims=True))
             assert np.all(np.abs(got - exp)[touched] <= 1e-5 * nrm[touched] + 1e-30)
