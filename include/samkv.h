@@ -176,6 +176,30 @@ samkv_status_t samkv_attn(samkv_handle_t h, const samkv_shape_t* shape, int32_t 
                           int32_t cache_capacity, int32_t* cache_len, const void* Q, int32_t T_q, const void* Kq,
                           const void* Vq, float scale, void* O, float* lse, void* stream);
 
+/* ---- scoring without any allocation ------------------------------------------------------ */
+
+/* (No counterpart in the paper: this entry point exists for deployment reasons only.)
+ * Same result as samkv_score, for callers that cannot call cudaMalloc or hand over a workspace:
+ * a serving engine whose memory pool already owns all of HBM, or a latency-critical section in
+ * which an allocation (which may synchronise the whole device) is not allowed.  It takes no handle.
+ * The personalised query vectors, the only scratch this step needs, live in a fixed array inside
+ * the library's device image: SAMKV_STATIC_SCORE_MAX_FLOATS fp32 values (1 MiB), held by every GPU
+ * that loads the library until the process exits.
+ *   - n_layers * batch * n_ctx * n_kv_heads * head_dim must not exceed SAMKV_STATIC_SCORE_MAX_FLOATS
+ *     (one layer of any configuration in this repository fits; call it layer by layer), otherwise
+ *     SAMKV_ERR_WORKSPACE is returned and nothing is launched.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array: two calls whose kernels can overlap on the GPU (different
+ *     streams, or several threads) race on it.  Order them on one stream.  The array keeps the last
+ *     call's contents; every element a call reads is rewritten by that call first, so no clearing
+ *     is needed.
+ *   - Calls no cudaMalloc / cudaFree or any other allocating routine.
+ * Arguments as in samkv_score (K, Q, Qloc, scores_out are caller-owned device pointers). */
+#define SAMKV_STATIC_SCORE_MAX_FLOATS (256 * 1024)
+samkv_status_t samkv_score_static(const samkv_shape_t* shape, const void* K, const void* Q, int32_t T_q,
+                                  const void* Qloc, int32_t T_loc, int32_t use_bias, float* scores_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

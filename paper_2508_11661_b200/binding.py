@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "SAMKV_OK", 1: "SAMKV_ERR_INVALID_ARG", 2: "SAMKV_ERR_UNSUPPO
 
 EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll_status", "samkv_status_string",
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
-           "samkv_attn"]
+           "samkv_attn", "samkv_score_static"]
 
 
 class SamkvError(RuntimeError):
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
     L.samkv_compact.argtypes = [vp, shp, vp, vp, vp, i32p, vp, vp, i32, vp, vp, vp]
     L.samkv_update.argtypes = [vp, shp, vp, vp, i32, vp, vp, i32, vp, vp, i32, vp]
     L.samkv_attn.argtypes = [vp, shp, i32, vp, vp, i32, vp, vp, i32, vp, vp, f32, vp, vp, vp]
+    L.samkv_score_static.argtypes = [shp, vp, vp, i32, vp, i32, i32, vp, vp]
     for name in EXPORTS:
         if name not in ("samkv_status_string", "samkv_workspace_bytes"):
             getattr(L, name).restype = ctypes.c_int
@@ -210,3 +211,11 @@ def samkv_attn(handle: Handle, shape: Shape, layer: int, Kc, Vc, cache_capacity:
     _check(lib().samkv_attn(handle.h, shape.ref(), layer, _ptr(Kc), _ptr(Vc), cache_capacity, _ptr(cache_len),
                             _ptr(Q), T_q, _ptr(Kq), _ptr(Vq), float(scale), _ptr(O), _ptr(lse), _stream()),
            "samkv_attn")
+
+
+def samkv_score_static(shape: Shape, K, Q, T_q: int, Qloc, T_loc: int, use_bias: int, scores_out):
+    """Scoring for callers that cannot allocate device memory (an engine whose pool owns all of HBM,
+    a section where cudaMalloc's implicit synchronisation is not acceptable): no handle, no workspace;
+    the scratch is a fixed 1 MiB array inside the library.  Calls sharing a GPU must not overlap."""
+    _check(lib().samkv_score_static(shape.ref(), _ptr(K), _ptr(Q), T_q, _ptr(Qloc), T_loc, int(use_bias),
+                                    _ptr(scores_out), _stream()), "samkv_score_static")

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsamkv.so")
-SOURCES = ["api.cu", "score.cu", "select.cu", "compact.cu", "attn.cu", "attn_mma.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "compact.cu", "attn.cu", "attn_mma.cu"]
 
 
 def nvcc_path() -> str:
@@ -50,7 +50,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}")
-    subprocess.check_call([nvcc_path(), "-shared", "-o", LIB_PATH] + objs)
+    subprocess.check_call([nvcc_path(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs)
     return LIB_PATH
 
 

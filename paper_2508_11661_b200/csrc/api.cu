@@ -113,6 +113,16 @@ inline samkv_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? SAMKV
 
 }  // namespace
 
+namespace samkv {
+// Shape validation + context tables for entry points that live in other files.
+samkv_status_t build_ctx_table(const samkv_shape_t* shape, CtxTable* ct) {
+  Layout lo;
+  samkv_status_t st = make_layout(shape, &lo);
+  if (st == SAMKV_OK) *ct = lo.ct;
+  return st;
+}
+}  // namespace samkv
+
 extern "C" {
 
 const char* samkv_status_string(samkv_status_t s) {
