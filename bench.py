@@ -68,7 +68,7 @@ def algorithmic_bytes(w, S: int, R: int, fusion: bool = True) -> dict:
 # clock sampling during the timed region
 # --------------------------------------------------------------------------------------------------
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -82,21 +82,33 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu_index)],
+                                          "-lms", "50", "-i", str(self.gpu_index)],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
+    def window_open(self):
+        import datetime
+        self.t0 = datetime.datetime.now()
+
+    def window_close(self):
+        import datetime
+        self.t1 = datetime.datetime.now()
+
     def stop(self) -> dict:
+        """Median SM clock and throttle reasons over the samples taken inside [window_open, window_close]
+        (all samples if the window caught none: the sampler's period is 50 ms)."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        rows = []
         try:
             with open(self.path) as f:
                 for line in f:
@@ -104,20 +116,24 @@ class ClockSampler:
                     if len(parts) < 9:
                         continue
                     try:
-                        sm.append(float(parts[1]))
-                        smax.append(float(parts[2]))
+                        ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                        rows.append((ts, float(parts[1]), float(parts[2]), parts[5:9]))
                     except ValueError:
                         continue
-                    for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
-                                         parts[5:9]):
-                        if val.lower().startswith("active"):
-                            reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons),
-                       samples=len(sm))
+        t0, t1 = getattr(self, "t0", None), getattr(self, "t1", None)
+        inside = [r for r in rows if t0 is not None and t1 is not None and t0 <= r[0] <= t1 + datetime.timedelta(milliseconds=60)]
+        use = inside if inside else rows
+        reasons = set()
+        for r in use:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if use:
+            out.update(sm_mhz=float(np.median([r[1] for r in use])), sm_max_mhz=float(max(r[2] for r in use)),
+                       reasons=sorted(reasons), samples=len(use), samples_in_timed_region=len(inside))
         return out
 
 
@@ -355,7 +371,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="samkv", choices=["samkv", "reference"])
     ap.add_argument("--workload", default="cfg2")
@@ -364,7 +380,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.warmup < 3 and args.impl == "samkv" and not args.layers:
+    profiling_case = bool(args.layers or args.batch)       # small captures under a profiler: keep launches few
+    if args.warmup < 3 and args.impl == "samkv" and not profiling_case:
         args.warmup = 3
 
     w = synth.CONFIGS[args.workload]
@@ -395,16 +412,17 @@ def main():
 
     pipe = Pipeline(w, dev, seed_offset=rank)
     pipe.prepare_recompute()
-    for _ in range(max(args.warmup, 3)):
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()            # started early: nvidia-smi needs a moment before its first sample
+    for _ in range(args.warmup):
         pipe.step()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
+    sampler.window_open()
     events = []
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
@@ -417,6 +435,7 @@ def main():
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
+    sampler.window_close()
     elapsed_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     if world > 1:
@@ -443,7 +462,7 @@ def main():
     pipeline_gbs = ab["total"] / (ms_per_step / 1e3) / 1e9
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "contexts": w.n_ctx,

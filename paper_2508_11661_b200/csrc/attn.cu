@@ -19,6 +19,10 @@ constexpr float kNegInf = -INFINITY;
 cudaError_t launch_attn_mma(const samkv_shape_t& s, int layer, const void* Kc, const void* Vc, int capacity,
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, cudaStream_t stream);
+cudaError_t launch_attn_tc(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
+                           const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
+                           float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
+                           cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Plan: how many packed rows a CTA takes and into how many KV splits a (batch, kv head) is cut.
@@ -28,21 +32,36 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
   AttnPlan p;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = T_q * G;
+  int ctas_per_sm, slots_per_tile, min_slots;
   if (s.dtype == SAMKV_BF16) {
-    p.rows_per_cta = rows > 64 ? 128 : (rows > 16 ? 64 : 16);
+    // >= 128 packed rows and d = 128: the tcgen05 kernel (128 rows per CTA, 2 CTAs per SM)
+    p.rows_per_cta = (rows >= 128 && s.head_dim == 128) ? 128 : (rows > 16 ? 64 : 16);
+    ctas_per_sm = rows > 16 ? 2 : 3;        // shared memory / registers of the attention kernels
+    slots_per_tile = 64;
+    min_slots = 256;
   } else {
     p.rows_per_cta = kSimtWarps;
+    ctas_per_sm = 8;
+    slots_per_tile = 64;
+    min_slots = 64;
   }
   const long long row_tiles = (rows + p.rows_per_cta - 1) / p.rows_per_cta;
   const long long base_ctas = (long long)s.batch * s.n_kv_heads * row_tiles;
-  const int min_slots = (s.dtype == SAMKV_BF16) ? 256 : 64;
-  long long want = (2LL * sm_count + base_ctas - 1) / (base_ctas > 0 ? base_ctas : 1);
-  long long max_by_len = capacity / min_slots;
-  if (max_by_len < 1) max_by_len = 1;
-  if (want > max_by_len) want = max_by_len;
-  if (want > 64) want = 64;
-  if (want < 1) want = 1;
-  p.n_splits = (int)want;
+  long long max_splits = capacity / min_slots;
+  if (max_splits > 64) max_splits = 64;
+  if (max_splits < 1) max_splits = 1;
+  // Pick the split count with the least (waves x work per CTA): a grid that spills a few CTAs into one
+  // more wave costs a whole wave, and every CTA pays a fixed prologue/epilogue (taken as 3 tiles).
+  const long long tiles = (capacity + slots_per_tile - 1) / slots_per_tile;
+  const long long slots = (long long)sm_count * ctas_per_sm;
+  long long best_n = 1, best_cost = -1;
+  for (long long n = 1; n <= max_splits; ++n) {
+    const long long tps = (tiles + n - 1) / n;
+    const long long waves = (base_ctas * n + slots - 1) / slots;
+    const long long cost = waves * (tps + 3);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
+  }
+  p.n_splits = (int)best_n;
   const size_t out_rows = (size_t)s.batch * T_q * s.n_q_heads;
   p.partial_bytes = p.n_splits > 1 ? out_rows * p.n_splits * ((size_t)s.head_dim * 4 + 8) : 0;
   return p;
@@ -249,8 +268,11 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int G = Hq / Hkv;
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
-    cudaError_t e = launch_attn_mma(s, layer, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
-                                    plan, stream);
+    cudaError_t e = (plan.rows_per_cta == 128)
+                        ? launch_attn_tc(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                                         plan, d_status, stream)
+                        : launch_attn_mma(s, layer, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o,
+                                          part_ml, plan, stream);
     if (e != cudaSuccess) return e;
   } else {
     const int row_tiles = (rows + kSimtWarps - 1) / kSimtWarps;

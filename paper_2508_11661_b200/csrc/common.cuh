@@ -63,7 +63,9 @@ cudaError_t launch_attn(const samkv_shape_t& s, int layer, void* Kc, void* Vc, i
 enum DeviceCheck : int {
   CHECK_OK = 0,
   CHECK_SEL_RANGE = 1,      // a selected unit id lies outside its context
-  CHECK_APPEND_CAPACITY = 2 // cache_len + T_q exceeds the cache capacity
+  CHECK_APPEND_CAPACITY = 2, // cache_len + T_q exceeds the cache capacity
+  CHECK_WAIT_TIMEOUT = 3,    // a bounded wait on an mbarrier ran out
+  CHECK_SMEM_ALIGNMENT = 4   // dynamic shared memory not aligned as the tensor-core tiles need
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
