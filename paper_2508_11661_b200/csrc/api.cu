@@ -32,6 +32,7 @@ samkv_status_t make_layout(const samkv_shape_t* s, Layout* lo) {
   if (s == nullptr || s->ctx_offsets == nullptr) return SAMKV_ERR_INVALID_ARG;
   if (s->n_layers < 1 || s->batch < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1) return SAMKV_ERR_INVALID_ARG;
   if (s->n_q_heads % s->n_kv_heads != 0) return SAMKV_ERR_INVALID_ARG;
+  if (s->n_q_heads / s->n_kv_heads > 32) return SAMKV_ERR_UNSUPPORTED;   // one warp per query head of a group
   if (s->n_ctx < 1) return SAMKV_ERR_INVALID_ARG;
   if (s->n_ctx > SAMKV_MAX_CTX) return SAMKV_ERR_UNSUPPORTED;
   if (s->head_dim != 64 && s->head_dim != 128) return SAMKV_ERR_UNSUPPORTED;
@@ -251,7 +252,7 @@ samkv_status_t samkv_score(samkv_handle_t handle, const samkv_shape_t* shape, co
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = launch_qhat(*shape, Q, T_q, Qloc, T_loc, use_bias, qhat, s);
   if (e != cudaSuccess) return SAMKV_ERR_CUDA;
-  return from_cuda(launch_score(*shape, lo.ct, K, qhat, scores_out, s));
+  return from_cuda(launch_score(*shape, lo.ct, K, qhat, scores_out, h->d_status, s));
 }
 
 samkv_status_t samkv_select(samkv_handle_t handle, const samkv_shape_t* shape, const float* scores,

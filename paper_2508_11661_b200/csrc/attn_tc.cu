@@ -11,7 +11,7 @@
 //                  its natural [slot][d] layout; O lives in tensor memory (128 columns) and is
 //                  rescaled there only when a row maximum grows by more than 2^8
 // MMAs are issued by one thread and complete on an mbarrier (tcgen05.commit).  K/V tiles are
-// staged by cp.async (rows past the visible range are zero-filled) in two stages; two CTAs share
+// staged by cp.async (rows past the visible range are zero-filled) in two-stage rings; two CTAs share
 // an SM so one CTA's softmax overlaps the other's MMAs.  Every wait is bounded: on a timeout the
 // kernel records a device check, frees its tensor memory and returns.
 #include <math.h>
@@ -215,19 +215,23 @@ attn_tc_kernel(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __rest
   }
   const __nv_bfloat16* kbase = Kc + (size_t)bh * capacity * kD;
   const __nv_bfloat16* vbase = Vc + (size_t)bh * capacity * kD;
-  auto load_tile = [&](int tile, int stage) {
+  // K and V tiles live in separate 2-stage rings so that K can be fetched one tile further ahead than V.
+  auto load_kv = [&](const __nv_bfloat16* gbase, uint32_t sbase, int tile, int stage) {
     const int j0 = tile * kBN;
     for (int i = tid; i < kBN * 16; i += kThreads) {
       const int r = i >> 4, c = i & 15;
       const bool ok = j0 + r < total;
       const size_t off = (size_t)(ok ? j0 + r : 0) * kD + c * 8;
-      const uint32_t d = stage * kTileBytes + (c >> 3) * (kBN * 128) + blk_off(r, c & 7);
-      cp_async16(sK + d, kbase + off, ok);
-      cp_async16(sV + d, vbase + off, ok);
+      cp_async16(sbase + stage * kTileBytes + (c >> 3) * (kBN * 128) + blk_off(r, c & 7), gbase + off, ok);
     }
   };
   const bool have_work = tile0 < tile1;
-  if (have_work) load_tile(tile0, 0);
+  if (have_work) {
+    load_kv(kbase, sK, tile0, 0);
+    load_kv(vbase, sV, tile0, 0);
+  }
+  cp_async_commit();
+  if (tile0 + 1 < tile1) load_kv(kbase, sK, tile0 + 1, 1);
   cp_async_commit();
 
   constexpr uint32_t kIdescS = instr_desc(kBM, kBN, false);
@@ -249,7 +253,7 @@ attn_tc_kernel(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __rest
     }
   };
 
-  cp_async_wait<0>();
+  cp_async_wait<1>();      // Q, K and V of the first tile (the second K tile may still be in flight)
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -273,7 +277,10 @@ attn_tc_kernel(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __rest
     failed = __any_sync(0xffffffffu, failed);
     phase ^= 1;
     tc_fence_after();
-    if (tile + 1 < tile1) load_tile(tile + 1, stage ^ 1);     // that stage's K and V are no longer in use
+    // K of this tile and V of the previous one are no longer in use: refill those stages now, a full
+    // iteration before the data is needed
+    if (tile + 2 < tile1) load_kv(kbase, sK, tile + 2, stage);
+    if (tile + 1 < tile1) load_kv(vbase, sV, tile + 1, stage ^ 1);
     cp_async_commit();
 
     // ---- softmax of this thread's row ----
@@ -281,12 +288,14 @@ attn_tc_kernel(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __rest
     tmem_ld32(lane_addr, s);
     tmem_ld32(lane_addr + 32, s + 32);
     const int j0 = tile * kBN;
+    if (j0 + kBN > vis) {        // only tiles that reach past this row's visible range need the mask
+#pragma unroll
+      for (int j = 0; j < kBN; ++j)
+        if (j0 + j >= vis) s[j] = -INFINITY;
+    }
     float mx = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < kBN; ++j) {
-      if (j0 + j >= vis) s[j] = -INFINITY;
-      mx = fmaxf(mx, s[j]);
-    }
+    for (int j = 0; j < kBN; ++j) mx = fmaxf(mx, s[j]);
     const float m_cand = fmaxf(m, mx * sl2);
     // keep the old reference maximum unless it would let P exceed 2^8 (or nothing has been seen yet)
     const bool grow = (m_cand - m > kRescaleThreshold) || (m == -INFINITY && m_cand > -INFINITY);
@@ -322,7 +331,7 @@ attn_tc_kernel(const __nv_bfloat16* __restrict__ Kc, const __nv_bfloat16* __rest
       }
       tmem_wait_st();
     }
-    cp_async_wait<0>();          // next tile's K/V have landed
+    cp_async_wait<1>();          // everything but this iteration's prefetch has landed: V of this tile, K of the next
     fence_proxy_async();         // P (st.shared) and K/V (cp.async) become visible to the tensor core
     tc_fence_before();
     __syncthreads();

@@ -39,7 +39,7 @@ struct samkv_ctx_impl {
 cudaError_t launch_qhat(const samkv_shape_t& s, const void* Q, int T_q, const void* Qloc, int T_loc, int use_bias,
                         float* qhat, cudaStream_t stream);
 cudaError_t launch_score(const samkv_shape_t& s, const CtxTable& ct, const void* K, const float* qhat, float* scores,
-                         cudaStream_t stream);
+                         int* d_status, cudaStream_t stream);
 cudaError_t launch_select(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const float* scores,
                           const int32_t* k_units_host, int max_units, int32_t* sel, int* d_status, cudaStream_t stream);
 cudaError_t launch_compact(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const void* K, const void* V,

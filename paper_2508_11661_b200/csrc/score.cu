@@ -4,25 +4,6 @@
 
 namespace samkv {
 
-// ------------------------------------------------------------------------------------------------
-// Block-wide sum of two values at once; blockDim.x is a multiple of 32 and at most 1024.
-// Fixed reduction tree => bitwise reproducible.
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ float2 block_sum2(float a, float b, float2* red) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    a += __shfl_xor_sync(0xffffffffu, a, o);
-    b += __shfl_xor_sync(0xffffffffu, b, o);
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  __syncthreads();  // protect `red` from the previous use
-  if (lane == 0) red[warp] = make_float2(a, b);
-  __syncthreads();
-  float2 r = make_float2(0.f, 0.f);
-  for (int i = 0; i < nw; ++i) { r.x += red[i].x; r.y += red[i].y; }
-  return r;
-}
-
 template <typename T>
 __device__ __forceinline__ float load_as_float(const T* p);
 template <>
@@ -30,181 +11,339 @@ __device__ __forceinline__ float load_as_float<float>(const float* p) { return *
 template <>
 __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Q_que = mean_t Q (Sec. 3.1), q_loc_j = mean_t Qloc_j, Eq. 1, then the mean over the G query heads
-// of a KV group.  One CTA per (layer, batch, kv head); thread e owns element e of the head dimension.
-// The sum over j != i is formed as (sum over all j) - (own term); fp32 throughout.
+// of a KV group.  One CTA per (layer, batch, kv head) with one warp per query head of the group; a lane
+// owns kEpl = d/32 consecutive elements, so the cosines need warp shuffles only (no block barriers
+// on the dependent chain).  The sum over j != i is formed as (sum over all j) - (own term); fp32.
 //   qhat [L*Bt, D, Hkv, d]
 // ------------------------------------------------------------------------------------------------
-template <typename T>
+template <typename T, int kEpl>
 __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc, float* __restrict__ qhat, int T_q,
-                            int T_loc, int Hq, int Hkv, int d, int D, int use_bias) {
+                            int T_loc, int Hq, int Hkv, int D, int use_bias) {
+  constexpr int d = kEpl * 32;
   extern __shared__ float smem[];
-  float* w = smem;                                        // [D] |cos| weights of the current query head
-  float2* red = reinterpret_cast<float2*>(smem + D + (D & 1));  // [32]
+  const int G = Hq / Hkv;
+  float* w_all = smem;                       // [G][D] |cos| weights
+  float* fold = smem + G * D;                // [G][d] per-head Q^_i of the context being folded
   const int h = blockIdx.x % Hkv;
   const size_t lb = blockIdx.x / Hkv;
-  const int e = threadIdx.x;
-  const int G = Hq / Hkv;
+  const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int hq = h * G + g;
   const bool bias = use_bias && Qloc != nullptr && D > 1;
-  float* out = qhat + (lb * D * Hkv + h) * d + e;          // + i * Hkv * d
-  const float inv_dm1 = bias ? 1.0f / (float)(D - 1) : 0.f;
+  float* w = w_all + g * D;
 
-  for (int g = 0; g < G; ++g) {
-    const int hq = h * G + g;
-    float qq = 0.f;
-    for (int t = 0; t < T_q; ++t) qq += load_as_float(Q + ((lb * T_q + t) * Hq + hq) * d + e);
-    qq = qq / (float)T_q;
-    float S = 0.f;
+  auto pooled = [&](const T* base, int T_n, size_t stride, float* out) {   // mean over T_n rows, summed in row order
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) out[i] = 0.f;
+    for (int t = 0; t < T_n; ++t) {
+#pragma unroll
+      for (int i = 0; i < kEpl; ++i) out[i] += load_as_float(base + t * stride + lane * kEpl + i);
+    }
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) out[i] = out[i] / (float)T_n;
+  };
+
+  float qq[kEpl], S[kEpl];
+  pooled(Q + (lb * T_q * Hq + hq) * d, T_q, (size_t)Hq * d, qq);
+#pragma unroll
+  for (int i = 0; i < kEpl; ++i) S[i] = 0.f;
+  if (bias) {
+    float na2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) na2 = fmaf(qq[i], qq[i], na2);
+    na2 = warp_sum(na2);
+    for (int j = 0; j < D; ++j) {
+      float ql[kEpl];
+      pooled(Qloc + ((lb * D + j) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql);
+      float dot = 0.f, nb2 = 0.f;
+#pragma unroll
+      for (int i = 0; i < kEpl; ++i) { dot = fmaf(qq[i], ql[i], dot); nb2 = fmaf(ql[i], ql[i], nb2); }
+      dot = warp_sum(dot);
+      nb2 = warp_sum(nb2);
+      const float wj = (na2 > 0.f && nb2 > 0.f) ? fabsf(dot) / (sqrtf(na2) * sqrtf(nb2)) : 0.f;
+      if (lane == 0) w[j] = wj;
+#pragma unroll
+      for (int i = 0; i < kEpl; ++i) S[i] = fmaf(wj, ql[i], S[i]);
+    }
+    __syncwarp();
+  }
+  const float inv_dm1 = bias ? 1.0f / (float)(D - 1) : 0.f;
+  float* out = qhat + (lb * D * Hkv + h) * d;            // + i * Hkv * d
+  for (int i0 = 0; i0 < D; ++i0) {
+    float val[kEpl];
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) val[i] = qq[i];
     if (bias) {
-      const float na2 = block_sum2(qq * qq, 0.f, red).x;
-      for (int j = 0; j < D; ++j) {
-        float ql = 0.f;
-        for (int t = 0; t < T_loc; ++t) ql += load_as_float(Qloc + (((lb * D + j) * T_loc + t) * Hq + hq) * d + e);
-        ql = ql / (float)T_loc;
-        const float2 r = block_sum2(qq * ql, ql * ql, red);
-        const float wj = (na2 > 0.f && r.y > 0.f) ? fabsf(r.x) / (sqrtf(na2) * sqrtf(r.y)) : 0.f;
-        if (e == 0) w[j] = wj;
-        S += wj * ql;
-      }
-      __syncthreads();
+      float ql[kEpl];
+      pooled(Qloc + ((lb * D + i0) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql);
+      const float wi = w[i0];
+#pragma unroll
+      for (int i = 0; i < kEpl; ++i) val[i] += (S[i] - wi * ql[i]) * inv_dm1;
     }
-    for (int i = 0; i < D; ++i) {
-      float val = qq;
-      if (bias) {
-        float ql = 0.f;
-        for (int t = 0; t < T_loc; ++t) ql += load_as_float(Qloc + (((lb * D + i) * T_loc + t) * Hq + hq) * d + e);
-        ql = ql / (float)T_loc;
-        val += (S - w[i] * ql) * inv_dm1;
-      }
-      float* o = out + (size_t)i * Hkv * d;
-      const float acc = (g == 0) ? val : (*o + val);
-      *o = (g == G - 1) ? acc / (float)G : acc;
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) fold[g * d + lane * kEpl + i] = val[i];
+    __syncthreads();
+    // mean over the G query heads of the group, summed in head order
+    for (int e = threadIdx.x; e < d; e += blockDim.x) {
+      float acc = fold[e];
+      for (int gg = 1; gg < G; ++gg) acc += fold[gg * d + e];
+      out[(size_t)i0 * Hkv * d + e] = acc / (float)G;
     }
-    __syncthreads();  // w[] is rewritten for the next query head
+    __syncthreads();
   }
 }
 
 cudaError_t launch_qhat(const samkv_shape_t& s, const void* Q, int T_q, const void* Qloc, int T_loc, int use_bias,
                         float* qhat, cudaStream_t stream) {
   const int blocks = s.n_layers * s.batch * s.n_kv_heads;
-  const size_t smem = (size_t)(s.n_ctx + (s.n_ctx & 1)) * sizeof(float) + 32 * sizeof(float2);
-  if (s.dtype == SAMKV_BF16)
-    qhat_kernel<__nv_bfloat16><<<blocks, s.head_dim, smem, stream>>>(
-        (const __nv_bfloat16*)Q, (const __nv_bfloat16*)Qloc, qhat, T_q, T_loc, s.n_q_heads, s.n_kv_heads, s.head_dim,
-        s.n_ctx, use_bias);
-  else
-    qhat_kernel<float><<<blocks, s.head_dim, smem, stream>>>((const float*)Q, (const float*)Qloc, qhat, T_q, T_loc,
-                                                             s.n_q_heads, s.n_kv_heads, s.head_dim, s.n_ctx, use_bias);
+  const int G = s.n_q_heads / s.n_kv_heads;
+  if (G > 32) return cudaErrorInvalidConfiguration;        // one warp per query head of a group
+  const size_t smem = (size_t)(G * s.n_ctx + G * s.head_dim) * sizeof(float);
+#define SAMKV_QHAT(T, EPL)                                                                                        \
+  qhat_kernel<T, EPL><<<blocks, G * 32, smem, stream>>>((const T*)Q, (const T*)Qloc, qhat, T_q, T_loc, s.n_q_heads, \
+                                                        s.n_kv_heads, s.n_ctx, use_bias)
+  if (s.dtype == SAMKV_BF16) {
+    if (s.head_dim == 128) SAMKV_QHAT(__nv_bfloat16, 4); else SAMKV_QHAT(__nv_bfloat16, 2);
+  } else {
+    if (s.head_dim == 128) SAMKV_QHAT(float, 4); else SAMKV_QHAT(float, 2);
+  }
+#undef SAMKV_QHAT
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
-// Streaming scorer.  A CTA owns a tile of kTile consecutive key rows of one context of one
-// (layer, batch, kv head) slab.  A row is kLanes 16-byte vectors; kLanes adjacent threads read one
-// row (fully coalesced), multiply with their slice of q_i held in registers and reduce with
-// shuffles.  All of a thread's loads are issued before the first use, so a CTA keeps
-// kTile * row_bytes (32 KB for bf16, d = 128) in flight.
+// Streaming scorer: one pass over every key row, s = <q_i, K_t>, unit score = mean over the unit.
+//
+// Persistent CTAs (two per SM) walk the list of tiles; a tile is up to 32 KB of consecutive key rows
+// of one context of one (layer, batch, kv head) slab, i.e. one contiguous run in HBM.  A producer
+// thread keeps a ring of kStages tiles in flight with bulk asynchronous copies (cp.async.bulk) that
+// complete on mbarriers, so the bytes in flight do not depend on how fast CTAs are launched or how
+// many registers the consumers hold.  Eight consumer warps read the tile from shared memory with
+// conflict-free 16-byte loads: kLanes adjacent threads own one row, multiply it with their slice
+// of q_i (registers) and reduce with shuffles.  Reduction order is fixed, so results are bitwise
+// reproducible.  Every mbarrier wait is bounded; a timeout is recorded as a device check.
 // ------------------------------------------------------------------------------------------------
-constexpr int kScoreThreads = 256;
-constexpr int kScoreTile = 128;
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kStreamThreads = kConsumers + 32;      // + one producer warp
+constexpr int kStages = 3;
+constexpr int kTileBytesMax = 32 * 1024;
+constexpr uint32_t kScoreSpinLimit = 1u << 22;
 
 struct TileTable {
-  int tile_off[SAMKV_MAX_CTX + 1];  // prefix sum of ceil(L_c / kScoreTile)
+  int tile_off[SAMKV_MAX_CTX + 1];  // prefix sum of ceil(L_c / rows per tile)
 };
 
-template <typename T, int kHeadDim>
-__global__ void __launch_bounds__(kScoreThreads)
-score_kernel(const T* __restrict__ K, const float* __restrict__ qhat, float* __restrict__ scores,
-             const __grid_constant__ CtxTable ct, const __grid_constant__ TileTable tt, int Hkv, int L_tot, int U_tot) {
-  constexpr int kPerVec = ElemTraits<T>::kPerVec;
-  constexpr int kLanes = kHeadDim / kPerVec;             // threads per row
-  constexpr int kRowsPerPass = kScoreThreads / kLanes;
-  constexpr int kPasses = kScoreTile / kRowsPerPass;
-  static_assert(kLanes <= 32 && kPasses >= 1, "row must fit in a warp");
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kScoreSpinLimit; ++i) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
 
-  __shared__ float s_tok[kScoreTile];
+template <typename T, int kHeadDim>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, float* __restrict__ scores,
+                    const __grid_constant__ CtxTable ct, const __grid_constant__ TileTable tt, int Hkv, int L_tot,
+                    int U_tot, long long total_tiles, int* __restrict__ d_status) {
+  constexpr int kPerVec = ElemTraits<T>::kPerVec;
+  constexpr int kRowBytes = kHeadDim * (int)sizeof(T);
+  constexpr int kRows = kTileBytesMax / kRowBytes;          // rows per tile
+  constexpr int kLanes = kHeadDim / kPerVec;                // threads per row
+  constexpr int kRowsPerPass = kConsumers / kLanes;
+  constexpr int kPasses = kRows / kRowsPerPass;
+  static_assert(kLanes <= 32 && kPasses >= 1 && kRows % 64 == 0, "tile shape");
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* tiles = smem_raw;                                        // kStages x 32 KB
+  float* s_tok = reinterpret_cast<float*>(smem_raw + kStages * kTileBytesMax);   // [kStages][kRows]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_tok + kStages * kRows);  // full[kStages], empty[kStages]
+  volatile int* s_fail = reinterpret_cast<volatile int*>(bars + 2 * kStages);
+  const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kStages);
+
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full0 + 8 * i), "r"(1) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty0 + 8 * i), "r"(kConsumerWarps) : "memory");
+    }
+    *s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
 
   const int tiles_per_slab = tt.tile_off[ct.n_ctx];
-  const int tile = blockIdx.x % tiles_per_slab;
-  const size_t slab = blockIdx.x / tiles_per_slab;         // (l * Bt + b) * Hkv + h
-  const int c = find_segment(tt.tile_off, ct.n_ctx, tile);
-  const int row0 = (tile - tt.tile_off[c]) * kScoreTile;    // first row of the tile inside its context
-  const int L_c = ct.ctx_off[c + 1] - ct.ctx_off[c];
-  const int rows = min(kScoreTile, L_c - row0);
+  const long long first = blockIdx.x, stride = gridDim.x;
 
-  const int lane = threadIdx.x % kLanes;
-  const int rsub = threadIdx.x / kLanes;
-  const int h = (int)(slab % Hkv);
-  const size_t lb = slab / Hkv;
+  // tile g -> (slab, context, first row inside the context, rows)
+  auto locate = [&](long long g, size_t& slab, int& c, int& row0, int& rows) {
+    slab = (size_t)(g / tiles_per_slab);
+    const int tile = (int)(g % tiles_per_slab);
+    c = find_segment(tt.tile_off, ct.n_ctx, tile);
+    row0 = (tile - tt.tile_off[c]) * kRows;
+    rows = min(kRows, ct.ctx_off[c + 1] - ct.ctx_off[c] - row0);
+  };
 
-  // this thread's slice of q_i
-  float q[kPerVec];
-  {
+  if (tid >= kConsumers) {
+    // ===== producer: one thread issues the bulk copies =====
+    if (tid == kConsumers) {
+      uint64_t policy;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+      long long n = 0;
+      bool ok = true;
+      for (long long g = first; g < total_tiles && ok; g += stride, ++n) {
+        const int stage = (int)(n % kStages);
+        const uint32_t round = (uint32_t)(n / kStages);
+        if (!mbar_wait_bounded(empty0 + 8 * stage, (round & 1) ^ 1)) { ok = false; break; }
+        size_t slab; int c, row0, rows;
+        locate(g, slab, c, row0, rows);
+        const uint32_t bytes = (uint32_t)rows * kRowBytes;
+        const T* src = K + (slab * L_tot + ct.ctx_off[c] + row0) * kHeadDim;
+        const uint32_t bar = full0 + 8 * stage;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+            ::"r"(smem_addr(tiles + stage * kTileBytesMax)), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+      }
+      // do not leave while a copy of ours may still be landing: wait (bounded) for the last copy of every stage
+      for (long long k = (n > kStages ? n - kStages : 0); k < n; ++k)
+        if (!mbar_wait_bounded(full0 + 8 * (int)(k % kStages), (uint32_t)((k / kStages) & 1))) ok = false;
+      if (!ok && d_status != nullptr) atomicMax(d_status, (int)CHECK_WAIT_TIMEOUT);
+    }
+    return;
+  }
+
+  // ===== consumers =====
+  const int lane = tid % kLanes;
+  const int rsub = tid / kLanes;
+  const int warp = tid >> 5;
+
+  auto load_q = [&](size_t slab, int c, float* q) {
+    const int h = (int)(slab % Hkv);
+    const size_t lb = slab / Hkv;
     const float* qp = qhat + ((lb * ct.n_ctx + c) * Hkv + h) * kHeadDim + lane * kPerVec;
 #pragma unroll
     for (int i = 0; i < kPerVec; i += 4) {
       const float4 v = *reinterpret_cast<const float4*>(qp + i);
       q[i] = v.x; q[i + 1] = v.y; q[i + 2] = v.z; q[i + 3] = v.w;
     }
-  }
+  };
 
-  const T* base = K + (slab * L_tot + ct.ctx_off[c] + row0) * kHeadDim + lane * kPerVec;
-  uint4 v[kPasses];
-#pragma unroll
-  for (int p = 0; p < kPasses; ++p) {
-    const int r = p * kRowsPerPass + rsub;
-    v[p] = (r < rows) ? ld_stream(base + (size_t)r * kHeadDim) : make_uint4(0, 0, 0, 0);
+  size_t slab; int c, row0, rows;
+  float q[kPerVec], q_next[kPerVec];
+  if (first < total_tiles) {
+    locate(first, slab, c, row0, rows);
+    load_q(slab, c, q);
   }
-#pragma unroll
-  for (int p = 0; p < kPasses; ++p) {
-    float f[kPerVec];
-    ElemTraits<T>::unpack(v[p], f);
-    float acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < kPerVec; ++i) acc = fmaf(f[i], q[i], acc);
-#pragma unroll
-    for (int o = kLanes / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) s_tok[p * kRowsPerPass + rsub] = acc;
-  }
-  __syncthreads();
+  long long n = 0;
+  for (long long g = first; g < total_tiles; g += stride, ++n) {
+    const int stage = (int)(n % kStages);
+    const uint32_t round = (uint32_t)(n / kStages);
+    // prefetch the next tile's q_i while this tile's bytes arrive
+    size_t slab_n = slab; int c_n = c, row0_n = row0, rows_n = rows;
+    const bool has_next = g + stride < total_tiles;
+    if (has_next) {
+      locate(g + stride, slab_n, c_n, row0_n, rows_n);
+      load_q(slab_n, c_n, q_next);
+    }
+    // A timeout is only recorded here; every consumer still reaches the named barrier below and they all
+    // leave together after it, so a failure can never strand a thread at a barrier.
+    if (!mbar_wait_bounded(full0 + 8 * stage, round & 1)) {
+      *s_fail = 1;
+      if (d_status != nullptr) atomicMax(d_status, (int)CHECK_WAIT_TIMEOUT);
+    }
 
-  // unit (block) scores: mean of the token scores of each unit, summed in token order
-  const int B = ct.block_size;
-  const int units = (rows + B - 1) >> ct.block_shift;
-  if ((int)threadIdx.x < units) {
-    const int a = threadIdx.x << ct.block_shift;
-    const int n = min(B, rows - a);
-    float sum = s_tok[a];
-    for (int i = 1; i < n; ++i) sum += s_tok[a + i];
-    scores[slab * U_tot + ct.unit_off[c] + (row0 >> ct.block_shift) + threadIdx.x] = (n == 1) ? sum : sum / (float)n;
+    const unsigned char* tile = tiles + stage * kTileBytesMax + lane * 16;
+    float* st = s_tok + stage * kRows;
+    uint4 v[kPasses];
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+      const int r = p * kRowsPerPass + rsub;
+      v[p] = (r < rows) ? *reinterpret_cast<const uint4*>(tile + (size_t)r * kRowBytes) : make_uint4(0, 0, 0, 0);
+    }
+    // the tile is in registers: hand the stage back to the producer
+    __syncwarp();
+    if ((tid & 31) == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * stage) : "memory");
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+      float f[kPerVec];
+      ElemTraits<T>::unpack(v[p], f);
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < kPerVec; ++i) acc = fmaf(f[i], q[i], acc);
+#pragma unroll
+      for (int o = kLanes / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) st[p * kRowsPerPass + rsub] = acc;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+    if (*s_fail) break;      // written only by consumers, before they arrived at the barrier: uniform
+
+    // unit (block) scores: mean of the token scores of each unit, summed in token order
+    const int Bsz = ct.block_size;
+    const int units = (rows + Bsz - 1) >> ct.block_shift;
+    if (tid < units) {
+      const int a = tid << ct.block_shift;
+      const int cnt = min(Bsz, rows - a);
+      float sum = st[a];
+      for (int i = 1; i < cnt; ++i) sum += st[a + i];
+      scores[slab * U_tot + ct.unit_off[c] + (row0 >> ct.block_shift) + tid] = (cnt == 1) ? sum : sum / (float)cnt;
+    }
+    (void)warp;
+    slab = slab_n; c = c_n; row0 = row0_n; rows = rows_n;
+#pragma unroll
+    for (int i = 0; i < kPerVec; ++i) q[i] = q_next[i];
   }
 }
 
 template <typename T, int kHeadDim>
 static cudaError_t launch_score_t(const samkv_shape_t& s, const CtxTable& ct, const void* K, const float* qhat,
-                                  float* scores, cudaStream_t stream) {
+                                  float* scores, int* d_status, cudaStream_t stream) {
+  constexpr int kRows = kTileBytesMax / (kHeadDim * (int)sizeof(T));
   TileTable tt;
   tt.tile_off[0] = 0;
   for (int c = 0; c < ct.n_ctx; ++c)
-    tt.tile_off[c + 1] = tt.tile_off[c] + (ct.ctx_off[c + 1] - ct.ctx_off[c] + kScoreTile - 1) / kScoreTile;
+    tt.tile_off[c + 1] = tt.tile_off[c] + (ct.ctx_off[c + 1] - ct.ctx_off[c] + kRows - 1) / kRows;
   const long long slabs = (long long)s.n_layers * s.batch * s.n_kv_heads;
-  const long long blocks = slabs * tt.tile_off[ct.n_ctx];
-  if (blocks == 0) return cudaSuccess;
-  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  score_kernel<T, kHeadDim><<<(unsigned)blocks, kScoreThreads, 0, stream>>>(
-      (const T*)K, qhat, scores, ct, tt, s.n_kv_heads, ct.ctx_off[ct.n_ctx], ct.unit_off[ct.n_ctx]);
+  const long long total_tiles = slabs * tt.tile_off[ct.n_ctx];
+  if (total_tiles == 0) return cudaSuccess;
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const size_t smem = (size_t)kStages * kTileBytesMax + (size_t)kStages * kRows * sizeof(float) + 2 * kStages * 8 + 16;
+  auto kern = score_stream_kernel<T, kHeadDim>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const long long grid = total_tiles < 2LL * sms ? total_tiles : 2LL * sms;
+  kern<<<(unsigned)grid, kStreamThreads, smem, stream>>>((const T*)K, qhat, scores, ct, tt, s.n_kv_heads,
+                                                         ct.ctx_off[ct.n_ctx], ct.unit_off[ct.n_ctx], total_tiles,
+                                                         d_status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_score(const samkv_shape_t& s, const CtxTable& ct, const void* K, const float* qhat, float* scores,
-                         cudaStream_t stream) {
+                         int* d_status, cudaStream_t stream) {
   if (s.dtype == SAMKV_BF16) {
-    if (s.head_dim == 128) return launch_score_t<__nv_bfloat16, 128>(s, ct, K, qhat, scores, stream);
-    return launch_score_t<__nv_bfloat16, 64>(s, ct, K, qhat, scores, stream);
+    if (s.head_dim == 128) return launch_score_t<__nv_bfloat16, 128>(s, ct, K, qhat, scores, d_status, stream);
+    return launch_score_t<__nv_bfloat16, 64>(s, ct, K, qhat, scores, d_status, stream);
   }
-  if (s.head_dim == 128) return launch_score_t<float, 128>(s, ct, K, qhat, scores, stream);
-  return launch_score_t<float, 64>(s, ct, K, qhat, scores, stream);
+  if (s.head_dim == 128) return launch_score_t<float, 128>(s, ct, K, qhat, scores, d_status, stream);
+  return launch_score_t<float, 64>(s, ct, K, qhat, scores, d_status, stream);
 }
 
 }  // namespace samkv

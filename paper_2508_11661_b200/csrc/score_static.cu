@@ -62,5 +62,6 @@ extern "C" samkv_status_t samkv_score_static(const samkv_shape_t* shape, const v
   // qhat_kernel writes every element of the range it uses before score_kernel reads it, so nothing
   // left over from an earlier call can leak into this one and nothing needs clearing.
   if (launch_qhat(*shape, Q, T_q, Qloc, T_loc, use_bias, qhat, s) != cudaSuccess) return SAMKV_ERR_CUDA;
-  return launch_score(*shape, ct, K, qhat, scores_out, s) == cudaSuccess ? SAMKV_OK : SAMKV_ERR_CUDA;
+  // no handle, hence no status word: the kernel's bounded waits cannot report here
+  return launch_score(*shape, ct, K, qhat, scores_out, nullptr, s) == cudaSuccess ? SAMKV_OK : SAMKV_ERR_CUDA;
 }
