@@ -163,15 +163,20 @@ score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, flo
   constexpr int kPerVec = ElemTraits<T>::kPerVec;
   constexpr int kRowBytes = kHeadDim * (int)sizeof(T);
   constexpr int kRows = kTileBytesMax / kRowBytes;          // rows per tile
-  constexpr int kLanes = kHeadDim / kPerVec;                // threads per row
+  constexpr int kChunks = kRowBytes / 16;                   // 16-byte chunks per row
+  constexpr int kLanes = kChunks / 2;                       // threads per row: chunks `lane` and `lane + kLanes`
   constexpr int kRowsPerPass = kConsumers / kLanes;
   constexpr int kPasses = kRows / kRowsPerPass;
-  static_assert(kLanes <= 32 && kPasses >= 1 && kRows % 64 == 0, "tile shape");
+  constexpr int kQBytes = kHeadDim * (int)sizeof(float);
+  static_assert(kLanes >= 1 && kLanes <= 32 && kPasses >= 1 && kRows % 64 == 0, "tile shape");
 
+  // shared memory: [tiles kStages x 32 KB][q kStages x kQBytes][token scores kStages x kRows][meta][barriers]
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* tiles = smem_raw;                                        // kStages x 32 KB
-  float* s_tok = reinterpret_cast<float*>(smem_raw + kStages * kTileBytesMax);   // [kStages][kRows]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_tok + kStages * kRows);  // full[kStages], empty[kStages]
+  unsigned char* tiles = smem_raw;
+  float* s_q = reinterpret_cast<float*>(smem_raw + kStages * kTileBytesMax);
+  float* s_tok = s_q + kStages * kHeadDim;
+  int4* s_meta = reinterpret_cast<int4*>(s_tok + kStages * kRows);          // {rows, score offset lo, hi, -}
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_meta + kStages);           // full[kStages], empty[kStages]
   volatile int* s_fail = reinterpret_cast<volatile int*>(bars + 2 * kStages);
   const uint32_t full0 = smem_addr(bars), empty0 = smem_addr(bars + kStages);
 
@@ -186,38 +191,37 @@ score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, flo
   }
   __syncthreads();
 
-  const int tiles_per_slab = tt.tile_off[ct.n_ctx];
   const long long first = blockIdx.x, stride = gridDim.x;
 
-  // tile g -> (slab, context, first row inside the context, rows)
-  auto locate = [&](long long g, size_t& slab, int& c, int& row0, int& rows) {
-    slab = (size_t)(g / tiles_per_slab);
-    const int tile = (int)(g % tiles_per_slab);
-    c = find_segment(tt.tile_off, ct.n_ctx, tile);
-    row0 = (tile - tt.tile_off[c]) * kRows;
-    rows = min(kRows, ct.ctx_off[c + 1] - ct.ctx_off[c] - row0);
-  };
-
   if (tid >= kConsumers) {
-    // ===== producer: one thread issues the bulk copies =====
+    // ===== producer: one thread locates each tile and issues its bulk copies (key rows + q_i) =====
     if (tid == kConsumers) {
+      const int tiles_per_slab = tt.tile_off[ct.n_ctx];
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
       long long n = 0;
       bool ok = true;
-      for (long long g = first; g < total_tiles && ok; g += stride, ++n) {
+      for (long long g = first; g < total_tiles; g += stride, ++n) {
         const int stage = (int)(n % kStages);
         const uint32_t round = (uint32_t)(n / kStages);
         if (!mbar_wait_bounded(empty0 + 8 * stage, (round & 1) ^ 1)) { ok = false; break; }
-        size_t slab; int c, row0, rows;
-        locate(g, slab, c, row0, rows);
+        const size_t slab = (size_t)(g / tiles_per_slab);           // (l * Bt + b) * Hkv + h
+        const int tile = (int)(g % tiles_per_slab);
+        const int c = find_segment(tt.tile_off, ct.n_ctx, tile);
+        const int row0 = (tile - tt.tile_off[c]) * kRows;           // first row of the tile inside its context
+        const int rows = min(kRows, ct.ctx_off[c + 1] - ct.ctx_off[c] - row0);
+        const long long out = (long long)slab * U_tot + ct.unit_off[c] + (row0 >> ct.block_shift);
+        s_meta[stage] = make_int4(rows, (int)(out & 0xffffffffLL), (int)(out >> 32), 0);
         const uint32_t bytes = (uint32_t)rows * kRowBytes;
         const T* src = K + (slab * L_tot + ct.ctx_off[c] + row0) * kHeadDim;
+        const float* qsrc = qhat + (((slab / Hkv) * ct.n_ctx + c) * Hkv + slab % Hkv) * kHeadDim;
         const uint32_t bar = full0 + 8 * stage;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes + kQBytes) : "memory");
         asm volatile(
             "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
             ::"r"(smem_addr(tiles + stage * kTileBytesMax)), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(s_q + stage * kHeadDim)), "l"(qsrc), "r"(kQBytes), "r"(bar) : "memory");
       }
       // do not leave while a copy of ours may still be landing: wait (bounded) for the last copy of every stage
       for (long long k = (n > kStages ? n - kStages : 0); k < n; ++k)
@@ -230,61 +234,57 @@ score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, flo
   // ===== consumers =====
   const int lane = tid % kLanes;
   const int rsub = tid / kLanes;
-  const int warp = tid >> 5;
 
-  auto load_q = [&](size_t slab, int c, float* q) {
-    const int h = (int)(slab % Hkv);
-    const size_t lb = slab / Hkv;
-    const float* qp = qhat + ((lb * ct.n_ctx + c) * Hkv + h) * kHeadDim + lane * kPerVec;
-#pragma unroll
-    for (int i = 0; i < kPerVec; i += 4) {
-      const float4 v = *reinterpret_cast<const float4*>(qp + i);
-      q[i] = v.x; q[i + 1] = v.y; q[i + 2] = v.z; q[i + 3] = v.w;
-    }
-  };
-
-  size_t slab; int c, row0, rows;
-  float q[kPerVec], q_next[kPerVec];
-  if (first < total_tiles) {
-    locate(first, slab, c, row0, rows);
-    load_q(slab, c, q);
-  }
   long long n = 0;
   for (long long g = first; g < total_tiles; g += stride, ++n) {
     const int stage = (int)(n % kStages);
     const uint32_t round = (uint32_t)(n / kStages);
-    // prefetch the next tile's q_i while this tile's bytes arrive
-    size_t slab_n = slab; int c_n = c, row0_n = row0, rows_n = rows;
-    const bool has_next = g + stride < total_tiles;
-    if (has_next) {
-      locate(g + stride, slab_n, c_n, row0_n, rows_n);
-      load_q(slab_n, c_n, q_next);
-    }
     // A timeout is only recorded here; every consumer still reaches the named barrier below and they all
     // leave together after it, so a failure can never strand a thread at a barrier.
     if (!mbar_wait_bounded(full0 + 8 * stage, round & 1)) {
       *s_fail = 1;
       if (d_status != nullptr) atomicMax(d_status, (int)CHECK_WAIT_TIMEOUT);
     }
-
+    const int4 meta = s_meta[stage];
+    const int rows = meta.x;
+    // this thread's two slices of q_i: elements of chunks `lane` and `lane + kLanes`
+    float q[2 * kPerVec];
+    {
+      const float* qs = s_q + stage * kHeadDim;
+#pragma unroll
+      for (int i = 0; i < kPerVec; i += 4) {
+        const float4 a = *reinterpret_cast<const float4*>(qs + lane * kPerVec + i);
+        const float4 b = *reinterpret_cast<const float4*>(qs + (lane + kLanes) * kPerVec + i);
+        q[i] = a.x; q[i + 1] = a.y; q[i + 2] = a.z; q[i + 3] = a.w;
+        q[kPerVec + i] = b.x; q[kPerVec + i + 1] = b.y; q[kPerVec + i + 2] = b.z; q[kPerVec + i + 3] = b.w;
+      }
+    }
     const unsigned char* tile = tiles + stage * kTileBytesMax + lane * 16;
     float* st = s_tok + stage * kRows;
-    uint4 v[kPasses];
+    uint4 v0[kPasses], v1[kPasses];
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
       const int r = p * kRowsPerPass + rsub;
-      v[p] = (r < rows) ? *reinterpret_cast<const uint4*>(tile + (size_t)r * kRowBytes) : make_uint4(0, 0, 0, 0);
+      if (r < rows) {
+        v0[p] = *reinterpret_cast<const uint4*>(tile + (size_t)r * kRowBytes);
+        v1[p] = *reinterpret_cast<const uint4*>(tile + (size_t)r * kRowBytes + kLanes * 16);
+      } else {
+        v0[p] = v1[p] = make_uint4(0, 0, 0, 0);
+      }
     }
-    // the tile is in registers: hand the stage back to the producer
+    // the tile (and q_i, meta) are in registers: hand the stage back to the producer
     __syncwarp();
     if ((tid & 31) == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8 * stage) : "memory");
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
-      float f[kPerVec];
-      ElemTraits<T>::unpack(v[p], f);
+      float f[kPerVec], g2[kPerVec];
+      ElemTraits<T>::unpack(v0[p], f);
+      ElemTraits<T>::unpack(v1[p], g2);
       float acc = 0.f;
 #pragma unroll
       for (int i = 0; i < kPerVec; ++i) acc = fmaf(f[i], q[i], acc);
+#pragma unroll
+      for (int i = 0; i < kPerVec; ++i) acc = fmaf(g2[i], q[kPerVec + i], acc);
 #pragma unroll
       for (int o = kLanes / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       if (lane == 0) st[p * kRowsPerPass + rsub] = acc;
@@ -300,12 +300,9 @@ score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, flo
       const int cnt = min(Bsz, rows - a);
       float sum = st[a];
       for (int i = 1; i < cnt; ++i) sum += st[a + i];
-      scores[slab * U_tot + ct.unit_off[c] + (row0 >> ct.block_shift) + tid] = (cnt == 1) ? sum : sum / (float)cnt;
+      const long long out = ((long long)meta.z << 32) | (unsigned int)meta.y;
+      scores[out + tid] = (cnt == 1) ? sum : sum / (float)cnt;
     }
-    (void)warp;
-    slab = slab_n; c = c_n; row0 = row0_n; rows = rows_n;
-#pragma unroll
-    for (int i = 0; i < kPerVec; ++i) q[i] = q_next[i];
   }
 }
 
@@ -325,7 +322,8 @@ static cudaError_t launch_score_t(const samkv_shape_t& s, const CtxTable& ct, co
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const size_t smem = (size_t)kStages * kTileBytesMax + (size_t)kStages * kRows * sizeof(float) + 2 * kStages * 8 + 16;
+  const size_t smem = (size_t)kStages * (kTileBytesMax + kHeadDim * sizeof(float) + kRows * sizeof(float) + 16) +
+                      2 * kStages * 8 + 16;
   auto kern = score_stream_kernel<T, kHeadDim>;
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
