@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsamkv.so")
-SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu"]
 
 
 def nvcc_path() -> str:
@@ -38,6 +38,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         common += ["-Xptxas", "-v"]
+    if os.environ.get("SAMKV_TRACE"):          # debugging aid: in-kernel timestamps in the attention kernel
+        common += ["-DSAMKV_TRACE"]
     procs = []
     for src in SOURCES:
         obj = os.path.join(build_dir, src.replace(".cu", ".o"))

@@ -19,10 +19,10 @@ constexpr float kNegInf = -INFINITY;
 cudaError_t launch_attn_mma(const samkv_shape_t& s, int layer, const void* Kc, const void* Vc, int capacity,
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, cudaStream_t stream);
-cudaError_t launch_attn_tc(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
-                           const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
-                           float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
-                           cudaStream_t stream);
+cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
+                            const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
+                            float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
+                            cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Plan: how many packed rows a CTA takes and into how many KV splits a (batch, kv head) is cut.
@@ -34,10 +34,12 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
   const int rows = T_q * G;
   int ctas_per_sm, slots_per_tile, min_slots;
   if (s.dtype == SAMKV_BF16) {
-    // >= 128 packed rows and d = 128: the tcgen05 kernel (128 rows per CTA, 2 CTAs per SM)
-    p.rows_per_cta = (rows >= 128 && s.head_dim == 128) ? 128 : (rows > 16 ? 64 : 16);
-    ctas_per_sm = rows > 16 ? 2 : 3;        // shared memory / registers of the attention kernels
-    slots_per_tile = 64;
+    // >= 128 packed rows and d = 128: the warp-specialised tcgen05 kernel (two 128-row tiles per CTA, one CTA
+    // per SM); otherwise mma.sync with 64 or 16 rows per CTA
+    const bool tc = rows >= 128 && s.head_dim == 128;
+    p.rows_per_cta = tc ? 256 : (rows > 16 ? 64 : 16);
+    ctas_per_sm = tc ? 1 : (rows > 16 ? 2 : 3);   // shared memory / registers of the attention kernels
+    slots_per_tile = tc ? 128 : 64;
     min_slots = 256;
   } else {
     p.rows_per_cta = kSimtWarps;
@@ -268,9 +270,9 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int G = Hq / Hkv;
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
-    cudaError_t e = (plan.rows_per_cta == 128)
-                        ? launch_attn_tc(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
-                                         plan, d_status, stream)
+    cudaError_t e = (plan.rows_per_cta == 256)
+                        ? launch_attn_tc2(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                                          plan, d_status, stream)
                         : launch_attn_mma(s, layer, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o,
                                           part_ml, plan, stream);
     if (e != cudaSuccess) return e;

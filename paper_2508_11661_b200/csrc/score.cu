@@ -42,6 +42,7 @@ __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc,
   auto pooled = [&](const T* base, int T_n, size_t stride, float* out) {   // mean over T_n rows, summed in row order
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) out[i] = 0.f;
+#pragma unroll 8
     for (int t = 0; t < T_n; ++t) {
 #pragma unroll
       for (int i = 0; i < kEpl; ++i) out[i] += load_as_float(base + t * stride + lane * kEpl + i);
@@ -59,6 +60,7 @@ __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc,
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) na2 = fmaf(qq[i], qq[i], na2);
     na2 = warp_sum(na2);
+#pragma unroll 4
     for (int j = 0; j < D; ++j) {
       float ql[kEpl];
       pooled(Qloc + ((lb * D + j) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql);
@@ -76,16 +78,20 @@ __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc,
   }
   const float inv_dm1 = bias ? 1.0f / (float)(D - 1) : 0.f;
   float* out = qhat + (lb * D * Hkv + h) * d;            // + i * Hkv * d
+  float ql_cur[kEpl], ql_nxt[kEpl];
+#pragma unroll
+  for (int i = 0; i < kEpl; ++i) ql_cur[i] = ql_nxt[i] = 0.f;
+  if (bias) pooled(Qloc + ((lb * D + 0) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql_cur);
   for (int i0 = 0; i0 < D; ++i0) {
+    // fetch the next context's local query before the barriers of this one
+    if (bias && i0 + 1 < D) pooled(Qloc + ((lb * D + i0 + 1) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql_nxt);
     float val[kEpl];
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) val[i] = qq[i];
     if (bias) {
-      float ql[kEpl];
-      pooled(Qloc + ((lb * D + i0) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql);
       const float wi = w[i0];
 #pragma unroll
-      for (int i = 0; i < kEpl; ++i) val[i] += (S[i] - wi * ql[i]) * inv_dm1;
+      for (int i = 0; i < kEpl; ++i) val[i] += (S[i] - wi * ql_cur[i]) * inv_dm1;
     }
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) fold[g * d + lane * kEpl + i] = val[i];
@@ -97,6 +103,8 @@ __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc,
       out[(size_t)i0 * Hkv * d + e] = acc / (float)G;
     }
     __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kEpl; ++i) ql_cur[i] = ql_nxt[i];
   }
 }
 
