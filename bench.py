@@ -37,6 +37,10 @@ HBM_NOMINAL_GBS = 8000.0
 HBM_FALLBACK_GBS = 6650.0
 
 # kernels each C-ABI call enqueues (memsets are not counted)
+# DRAM bytes per scored key row of score_stream_kernel, from the ncu capture summarised in
+# profiles/score_stream_kernel_cfg2_2layers.md (dram read + write of one launch / rows of that launch);
+# traffic grows in proportion to the rows (no reuse), so a full launch is rows x this figure.
+SCORE_KERNEL_DRAM_BYTES_PER_ROW = 260.0
 KERNELS_PER_CALL = {"score": 2, "select": 1, "compact": 1, "update": 1, "attn_append_split": 3}
 
 
@@ -368,6 +372,28 @@ def run_reference(args, w):
 
 
 # --------------------------------------------------------------------------------------------------
+# multi-GPU host logic (no data-path collective: every rank owns an independent request batch)
+# --------------------------------------------------------------------------------------------------
+def rank_workload(w, rank: int):
+    """Weak scaling: rank r processes its own batch of the same shape, generated from seed + r."""
+    return w.replace(seed=w.seed + rank)
+
+
+def max_over_ranks(elapsed_ms: float, device) -> float:
+    """The job's step time is the slowest rank's device time."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(elapsed_ms)
+    t = torch.tensor([elapsed_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(w, world: int, ms_per_step: float) -> float:
+    """Whole-job context tokens per second: every rank pushes batch x L_tot tokens through all layers."""
+    return w.batch * w.l_tot * world / (ms_per_step / 1e3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,7 +436,7 @@ def main():
     if world > 1:
         dist.barrier()
 
-    pipe = Pipeline(w, dev, seed_offset=rank)
+    pipe = Pipeline(rank_workload(w, rank), dev)
     pipe.prepare_recompute()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -438,10 +464,7 @@ def main():
     sampler.window_close()
     elapsed_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dev)
     status = pipe.B.samkv_poll_status(pipe.handle)
     if status != 0:
         raise RuntimeError(f"device-side check failed during the benchmark (status {status})")
@@ -453,8 +476,7 @@ def main():
             phase_ms[n1] = phase_ms.get(n1, 0.0) + a.elapsed_time(b) / args.steps
 
     ms_per_step = elapsed_ms / args.steps
-    tokens_per_step = w.batch * w.l_tot * world
-    value = tokens_per_step / (ms_per_step / 1e3)
+    value = job_throughput(w, world, ms_per_step)
     peaks, peak_kind = measured_peaks()
     hbm_peak = float(peaks.get("hbm_gbs", HBM_FALLBACK_GBS))
     ab = algorithmic_bytes(w, pipe.S, pipe.R, fusion=True)
@@ -478,7 +500,10 @@ def main():
         "roofline": {"kernel": "score_kernel (with the pooled-query kernel that precedes it in samkv_score)", "bound": "hbm",
                      "achieved": score_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": score_gbs / hbm_peak, "frac_of_nominal_8tbs": score_gbs / HBM_NOMINAL_GBS,
-                     "algorithmic_bytes_per_launch": ab["score"], "traffic": None},
+                     "algorithmic_bytes_per_launch": ab["score"],
+                     "traffic": (SCORE_KERNEL_DRAM_BYTES_PER_ROW * w.n_layers * w.batch * w.n_kv_heads * w.l_tot
+                                 if (w.dtype == "bf16" and w.head_dim == 128) else None),
+                     "traffic_note": "ncu dram read+write of a 2-layer launch scaled by rows (profiles/)"},
         "gpu_launches": pipe.launches_per_step() * args.steps,
         "clocks": clocks,
     }
