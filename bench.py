@@ -64,8 +64,10 @@ def algorithmic_bytes(w, S: int, R: int, fusion: bool = True) -> dict:
     gather = slabs * S * row * 4                          # read K,V rows, write Kc,Vc rows
     upd = w.n_layers * w.batch * R * w.n_kv_heads * row * (6 if fusion else 4)
     attn = slabs * (S + w.q_tokens) * row * 2             # attention reads Kc,Vc (cache + chunk)
-    return {"score": score, "compact": gather, "update": upd, "attn": attn,
-            "total": score + gather + upd + attn}
+    # decode step i reads the cache as it stands then: S + T_q + i slots (+ its own row)
+    dec = sum(slabs * (S + w.q_tokens + i + 1) * row * 2 for i in range(w.decode_steps))
+    return {"score": score, "compact": gather, "update": upd, "attn": attn, "decode": dec,
+            "total": score + gather + upd + attn + dec}
 
 
 # --------------------------------------------------------------------------------------------------
@@ -156,7 +158,7 @@ class Pipeline:
         self.shape = B.Shape.from_workload(w)
         self.k_units = B.samkv_budget_units(self.shape, w.budget_bp)
         _, self.U_tot, self.S = B.samkv_layout(self.shape, self.k_units)
-        self.capacity = self.S + w.q_tokens
+        self.capacity = self.S + w.q_tokens + w.decode_steps
         L, Bt, Hkv, d = w.n_layers, w.batch, w.n_kv_heads, w.head_dim
         self.handle = B.Handle(self.shape, w.q_tokens, self.capacity)
         self.scores = torch.empty((L, Bt, Hkv, self.U_tot), dtype=torch.float32, device=device)
@@ -169,6 +171,14 @@ class Pipeline:
         self.R = 0
         self.tok_ids = self.Knew = self.Vnew = None
         self.t_loc = self.inp["Qloc"].shape[3]
+        self.decode_graph = None
+        if w.decode_steps > 0:      # one query token per step and batch element, appended to the compact cache
+            g = torch.Generator(device=device).manual_seed(w.seed + 99)
+            n = w.decode_steps
+            self.dq = torch.randn((n, Bt, 1, w.n_q_heads, d), generator=g, device=device).to(w.torch_dtype)
+            self.dk = torch.randn((n, Bt, 1, Hkv, d), generator=g, device=device).to(w.torch_dtype)
+            self.dv = torch.randn((n, Bt, 1, Hkv, d), generator=g, device=device).to(w.torch_dtype)
+            self.dO = torch.empty_like(self.dq)
 
     def prepare_recompute(self):
         """Recompute list: R = 15 % of the kept tokens, drawn from what KV head 0 kept (needs one selection pass)."""
@@ -215,12 +225,41 @@ class Pipeline:
             B.samkv_attn(self.handle, self.shape, l, self.Kc, self.Vc, self.capacity, self.cache_len, inp["Qa"][l],
                          w.q_tokens, inp["Kq"][l], inp["Vq"][l], 0.0, self.O[l])
         mark("attn")
+        if w.decode_steps > 0:
+            self.decode()
+            mark("decode")
+
+    def decode_eager(self):
+        B, w = self.B, self.w
+        for l in range(w.n_layers):
+            for i in range(w.decode_steps):
+                B.samkv_attn(self.handle, self.shape, l, self.Kc, self.Vc, self.capacity, self.cache_len, self.dq[i], 1,
+                             self.dk[i], self.dv[i], 0.0, self.dO[i])
+
+    def decode(self):
+        """The decode loop is launch-bound when driven from Python, so it is captured once in a CUDA graph
+        (cache_len lives on the device, so the same graph is valid for every replay) and replayed."""
+        if self.decode_graph is None:
+            torch.cuda.synchronize()
+            saved = self.cache_len.clone()
+            side = torch.cuda.Stream(device=self.dev)
+            side.wait_stream(torch.cuda.current_stream())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    self.decode_eager()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            self.cache_len.copy_(saved)
+            self.decode_graph = g
+        self.decode_graph.replay()
 
     def launches_per_step(self) -> int:
         n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + KERNELS_PER_CALL["compact"]
         if self.R > 0:
             n += KERNELS_PER_CALL["update"]
-        return n + self.w.n_layers * KERNELS_PER_CALL["attn_append_split"]
+        n += self.w.n_layers * KERNELS_PER_CALL["attn_append_split"]
+        return n + self.w.n_layers * self.w.decode_steps * KERNELS_PER_CALL["attn_append_split"]
 
 
 def e2e_steps(pipe: Pipeline, steps: int, warmup: int):
@@ -403,6 +442,7 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling captures of a small case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling captures of a small case)")
+    ap.add_argument("--budget-bp", type=int, default=0, help="override the sequence budget (basis points)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -415,6 +455,8 @@ def main():
         w = w.replace(n_layers=args.layers)
     if args.batch:
         w = w.replace(batch=args.batch)
+    if args.budget_bp:
+        w = w.replace(budget_bp=args.budget_bp)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -496,7 +538,7 @@ def main():
         "pipeline": {"algorithmic_gb_per_step": ab["total"] / 1e9, "achieved_gbs": pipeline_gbs,
                      "frac_of_measured_copy_peak": pipeline_gbs / hbm_peak, "frac_of_nominal_8tbs": pipeline_gbs / HBM_NOMINAL_GBS,
                      "phase_ms": phase_ms,
-                     "phase_gbs": {k: ab[k] / (phase_ms[k] / 1e3) / 1e9 for k in ("score", "compact", "update", "attn") if phase_ms.get(k, 0) > 0}},
+                     "phase_gbs": {k: ab[k] / (phase_ms[k] / 1e3) / 1e9 for k in ("score", "compact", "update", "attn", "decode") if phase_ms.get(k, 0) > 0}},
         "roofline": {"kernel": "score_kernel (with the pooled-query kernel that precedes it in samkv_score)", "bound": "hbm",
                      "achieved": score_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": score_gbs / hbm_peak, "frac_of_nominal_8tbs": score_gbs / HBM_NOMINAL_GBS,
@@ -508,7 +550,10 @@ def main():
         "clocks": clocks,
     }
 
-    if rank == 0 and not args.no_e2e:
+    if w.decode_steps > 0:
+        line["decode"] = {"steps": w.decode_steps, "us_per_step": phase_ms["decode"] * 1e3 / w.decode_steps / w.n_layers,
+                          "achieved_gbs": ab["decode"] / (phase_ms["decode"] / 1e3) / 1e9, "launch": "cuda graph"}
+    if rank == 0 and not args.no_e2e and w.decode_steps == 0:
         try:
             import psutil
             free = psutil.virtual_memory().available

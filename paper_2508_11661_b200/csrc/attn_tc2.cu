@@ -55,7 +55,7 @@ constexpr float kRescaleThreshold = 8.0f;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // barrier slots (8 bytes each) inside the barrier block
-enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, KV_TMA = 8, S_FULL = 9, P_READY = 11, O_FINAL = 13, N_BARS = 14 };
+enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, KV_TMA = 8, S_FULL = 9, P_READY = 11, O_FINAL = 13, Q_READY = 14, N_BARS = 15 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
@@ -246,6 +246,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
     mbar_init(bar(KV_TMA), 1);
     mbar_init(bar(O_FINAL), 1);
+    mbar_init(bar(Q_READY), kSoftmaxWarps);
     for (int q = 0; q < 2; ++q) {
       mbar_init(bar(S_FULL + q), 1);
       mbar_init(bar(P_READY + q), 4);     // one arrival per softmax warp of the tile
@@ -258,7 +259,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // Q tiles: cp.async by the softmax warps, rows beyond the chunk zero-filled
+  tc_fence_before();
+  __syncthreads();            // barriers initialised, tensor memory allocated: the roles part ways here
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  // Q tiles: cp.async by the softmax warps (rows beyond the chunk zero-filled) while the loader already
+  // streams the first K/V tiles; the MMA thread waits for Q_READY before its first product
   if (warp < kSoftmaxWarps) {
     for (int i = tid; i < 2 * kBM * 16; i += kSoftmaxWarps * 32) {
       const int r = i >> 4, c = i & 15;                       // r in [0, 256)
@@ -271,11 +278,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(Q_READY));
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *s_tmem;
 
   if (warp == kLoadWarp) {
     // ================= loader: K ring and V ring =================
@@ -338,6 +343,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           mma_ts(tmem + kTmemO + q * kD, tmem + q * kBN + ks * 8, b0 + ((ks * 16 * 128) >> 4), kIdescO,
                  accumulate | (ks > 0));
       };
+      mbar_wait(bar(Q_READY), 0, s_fail);
       mbar_wait(bar(K_FULL + 0), 0, s_fail);
       tc_fence_after();
       for (int q = 0; q < n_q; ++q) issue_s(q, 0);
