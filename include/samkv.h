@@ -134,7 +134,10 @@ samkv_status_t samkv_select(samkv_handle_t h, const samkv_shape_t* shape, const 
 
 /* Compaction (Sec. 3.2: initial + selected + local rows joined in their original order).
  *   Kc[l,b,h,slot,:] = K[l,b,h,tok(slot),:], same for V; slots run over (context, token) ascending.
- *   K, V      [L, Bt, Hkv, L_tot, d]
+ *   K, V      [L, Bt, Hkv, L_tot, d].  V (only V) may also be a pointer into PINNED HOST memory that the
+ *             device can address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel
+ *             then pulls just the kept V rows across the bus, so only the kept share of V is ever loaded
+ *             to the GPU (the paper's "sequence ratio", Table 1); K is read on the device by samkv_score anyway
  *   sel       int32 [L, Bt, Hkv, S_u] as written by samkv_select; k_units host [n_ctx]
  *   Kc, Vc    [L, Bt, Hkv, cache_capacity, d]; slots >= S are left untouched
  *   cache_len int32 [L, Bt], set to S (the number of kept tokens)

@@ -109,11 +109,11 @@ def _check(status: int, where: str):
         raise SamkvError(status, where)
 
 
-def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+def _ptr(t: Optional[torch.Tensor], allow_pinned_host: bool = False) -> Optional[int]:
     if t is None:
         return None
-    if not t.is_cuda:
-        raise ValueError("expected a CUDA tensor")
+    if not t.is_cuda and not (allow_pinned_host and t.is_pinned()):
+        raise ValueError("expected a CUDA tensor" + (" or a pinned host tensor" if allow_pinned_host else ""))
     if not t.is_contiguous():
         raise ValueError("expected a contiguous tensor")
     return t.data_ptr()
@@ -196,7 +196,9 @@ def samkv_select(handle: Handle, shape: Shape, scores, k_units: Sequence[int], s
 
 def samkv_compact(handle: Handle, shape: Shape, K, V, sel, k_units: Sequence[int], Kc, Vc, cache_capacity: int,
                   cache_len, inv_map=None):
-    _check(lib().samkv_compact(handle.h, shape.ref(), _ptr(K), _ptr(V), _ptr(sel), _i32_array(k_units), _ptr(Kc),
+    # V may live in pinned host memory: the gather then reads only the kept rows across the bus
+    _check(lib().samkv_compact(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(sel),
+                               _i32_array(k_units), _ptr(Kc),
                                _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()), "samkv_compact")
 
 

@@ -253,3 +253,23 @@ def test_append_past_capacity_is_reported_not_fatal():
     Og2, _ = run.attn(0, inp["Qa"][0])                              # cache-only attention still works
     check_attention(w, run.Kc[0, 0], run.Vc[0, 0], run.S, inp["Qa"][0, 0], None, None, Og2[0])
     assert torch.equal(Og, Og2)
+
+
+def test_compact_gathers_v_rows_from_pinned_host_memory():
+    """V may stay in pinned host memory; only the kept rows cross the bus.  Same bits as with V on the device."""
+    w = synth.CONFIGS["cfg1"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    Kc_dev, Vc_dev = run.Kc.clone(), run.Vc.clone()
+    V_host = inp["V"].cpu().pin_memory()
+    run.Kc.zero_(); run.Vc.zero_()
+    B.samkv_compact(run.handle, run.shape, inp["K"], V_host, run.sel, run.k_units, run.Kc, run.Vc, run.capacity,
+                    run.cache_len, run.inv_map)
+    torch.cuda.synchronize()
+    assert torch.equal(run.Kc, Kc_dev) and torch.equal(run.Vc, Vc_dev)
+    check_compact(w, run, 0, 0, run.sel[0, 0].cpu().numpy())
+    with pytest.raises(ValueError):                                   # pageable host memory is refused by the binding
+        B.samkv_compact(run.handle, run.shape, inp["K"], inp["V"].cpu(), run.sel, run.k_units, run.Kc, run.Vc,
+                        run.capacity, run.cache_len, run.inv_map)
+    assert run.poll() == 0
