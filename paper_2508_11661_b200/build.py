@@ -38,8 +38,6 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         common += ["-Xptxas", "-v"]
-    if os.environ.get("SAMKV_TRACE"):          # debugging aid: in-kernel timestamps in the attention kernel
-        common += ["-DSAMKV_TRACE"]
     procs = []
     for src in SOURCES:
         obj = os.path.join(build_dir, src.replace(".cu", ".o"))

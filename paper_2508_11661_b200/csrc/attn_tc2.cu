@@ -24,15 +24,6 @@
 #include "common.cuh"
 
 namespace samkv {
-#ifdef SAMKV_TRACE
-__device__ long long g_trace[8192];
-#define TRACE(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_trace[(slot)] = clock64(); } while (0)
-extern "C" int samkv_debug_trace(long long* host_out, int n) {
-  return (int)cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * n);
-}
-#else
-#define TRACE(slot) do {} while (0)
-#endif
 namespace tc2 {
 
 constexpr int kBM = 128, kBN = 128, kD = 128;
@@ -350,19 +341,15 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       mma_commit(bar(K_EMPTY + 0));
       for (int j = 0; j < nt; ++j) {
         const int s = j % kStages, s1 = (j + 1) % kStages;
-        TRACE(4096 + j * 8 + 0);
         mbar_wait(bar(V_FULL + s), (uint32_t)((j / kStages) & 1), s_fail);
         if (j + 1 < nt) mbar_wait(bar(K_FULL + s1), (uint32_t)(((j + 1) / kStages) & 1), s_fail);
-        TRACE(4096 + j * 8 + 1);
         for (int q = 0; q < n_q; ++q) {
           // P_q of this tile is in tensor memory (and S_q has been consumed): O_q += P_q V, then S_q of the
           // next tile may overwrite the same columns (the tensor pipe executes in issue order)
           mbar_wait(bar(P_READY + q), (uint32_t)(j & 1), s_fail);
           tc_fence_after();
-          TRACE(4096 + j * 8 + 2 + 2 * q);
           issue_pv(q, s, j > 0);
           if (j + 1 < nt) issue_s(q, s1);
-          TRACE(4096 + j * 8 + 3 + 2 * q);
         }
         mma_commit(bar(V_EMPTY + s));                            // every MMA so far finished: V_j (and K_{j+1}) are free
         if (j + 1 < nt) mma_commit(bar(K_EMPTY + s1));
@@ -385,10 +372,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (active) {
       for (int j = 0; j < nt; ++j) {
         // S_q(j) complete; so is every earlier MMA, in particular P_q(j-1) V, hence O_q and the P columns are ours
-        if (tid == 0) TRACE(j * 8 + 0);
         mbar_wait_warp(bar(S_FULL + q), (uint32_t)(j & 1), s_fail);
         tc_fence_after();
-        if (tid == 0) TRACE(j * 8 + 1);
         const int j0 = (tile0 + j) * kBN;
         const bool masked = j0 + kBN > vis;
         // pass 1: row maximum (two loads in flight)
@@ -410,7 +395,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           }
         }
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-        if (tid == 0) TRACE(j * 8 + 2);
         const float m_cand = fmaxf(m, mx * sl2);
         const bool grow = (m_cand - m > kRescaleThreshold) || (m == -INFINITY && m_cand > -INFINITY);
         const float m_use = grow ? m_cand : m;
@@ -457,7 +441,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_READY + q));
-        if (tid == 0) TRACE(j * 8 + 3);
       }
       if (nt > 0) {
         mbar_wait_warp(bar(O_FINAL), 0, s_fail);
