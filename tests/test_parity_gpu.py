@@ -273,3 +273,56 @@ def test_compact_gathers_v_rows_from_pinned_host_memory():
         B.samkv_compact(run.handle, run.shape, inp["K"], inp["V"].cpu(), run.sel, run.k_units, run.Kc, run.Vc,
                         run.capacity, run.cache_len, run.inv_map)
     assert run.poll() == 0
+
+
+def test_many_contexts_and_raw_local_query_rows():
+    """128 contexts (the library's maximum), ragged lengths, raw local Q rows (T_loc = n_local) in bf16, G = 8."""
+    g = torch.Generator().manual_seed(3)
+    lens = tuple(int(x) for x in torch.randint(40, 90, (128,), generator=g))
+    w = synth.Workload("many_ctx", 1, 2, 16, 2, 128, "bf16", lens, 4, budget_bp=2500, block_size=1, n_init=4, n_local=8,
+                       t_loc=8, rope_base=10000.0, seed=31)
+    full_check(w)
+    shape = B.Shape.from_workload(w.replace(ctx_lens=lens + (50,)))
+    with pytest.raises(B.SamkvError) as e:                              # 129 contexts: refused, not truncated
+        B.samkv_budget_units(shape, 1500)
+    assert e.value.status == 2
+
+
+def test_large_context_uses_block_wide_select_and_head_dim_64_prefill():
+    """One context of 20 000 tokens (block-wide radix select, several passes over shared memory) next to a short
+    one; head_dim 64 with 160 packed rows goes through the 64-row mma.sync tiling."""
+    w = synth.Workload("big_ctx", 1, 1, 8, 2, 64, "bf16", (20000, 300), 20, budget_bp=1000, block_size=1, n_init=16,
+                       n_local=32, t_loc=1, rope_base=10000.0, seed=41)
+    run, _ = full_check(w)
+    assert run.S == 2000 + 48
+
+
+def test_paper_block_settings_on_decode_shape():
+    """Block size 64 with 1 initial and 2 local blocks (the paper's settings) on a reduced cfg3: block-mean scores,
+    block selection, then prefill chunk and a few decode steps."""
+    w = synth.CONFIGS["cfg3"].replace(name="cfg3_b64", batch=2, ctx_lens=(2048, 1999, 1024), block_size=64, n_init=64,
+                                      n_local=128, budget_bp=2500, decode_steps=3)
+    run, _ = full_check(w)
+    inp = run.inp
+    g = torch.Generator().manual_seed(19)
+    n = run.S + w.q_tokens
+    ref = [(to_f64(run.Kc[0, b]), to_f64(run.Vc[0, b])) for b in range(w.batch)]
+    for step in range(w.decode_steps):
+        q = torch.randn((w.batch, 1, w.n_q_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        kq = torch.randn((w.batch, 1, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        vq = torch.randn((w.batch, 1, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        Os, _ = run.attn(0, q, kq, vq)
+        for b in range(w.batch):
+            out, _, K2, V2, _ = O.attention(ref[b][0], ref[b][1], n, to_f64(q[b]), to_f64(kq[b]), to_f64(vq[b]))
+            ref[b] = (K2, V2)
+            assert np.abs(to_f64(Os[b]) - out).max() <= 2e-2
+        n += 1
+    assert run.poll() == 0
+
+
+def test_context_beyond_shared_memory_is_refused():
+    w = synth.Workload("huge_ctx", 1, 1, 4, 2, 64, "f32", (60000,), 2, n_init=4, n_local=8, t_loc=1, seed=5)
+    shape = B.Shape.from_workload(w)
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_budget_units(shape, 1500)                               # more units in one context than the select kernel holds
+    assert e.value.status == 2
