@@ -422,3 +422,125 @@ def sparsify(K, V, Q, Qloc, ctx_offsets, B, n_init, n_local, k_units, use_bias=T
     sel = select_units(u, ctx_offsets, B, n_init, n_local, k_units)
     Kc, Vc, S, inv = compact(K, V, sel, ctx_offsets, B, capacity)
     return dict(Q_que=Q_que, q_loc=q_loc, Qhat=Qhat, q=q, s=s, u=u, sel=sel, Kc=Kc, Vc=Vc, cache_len=S, inv_map=inv)
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.2, Eq. 2 and Eq. 3: dynamic Top-P from anchor / max / min scores, then the
+# cross-context Top-K.  (Widening beyond the fixed-budget selection above.)
+# --------------------------------------------------------------------------------------
+def anchor_score(u_row: np.ndarray, c: int, ctx_offsets, B: int, n_init: int, n_local: int) -> float:
+    """s_anc of context c: the anchor vector is read as the mean key over the protected
+    (initial + local) tokens, so its score is the token-count-weighted mean of the protected
+    units' scores (unit scores are means over their tokens)."""
+    nb, unit_off = unit_layout(ctx_offsets, B)
+    L_c = int(ctx_offsets[c + 1]) - int(ctx_offsets[c])
+    tot, cnt = 0.0, 0
+    for m in protected_units(L_c, B, n_init, n_local):
+        n_tok = min((m + 1) * B, L_c) - m * B
+        tot += float(u_row[unit_off[c] + m]) * n_tok
+        cnt += n_tok
+    return tot / cnt if cnt else 0.0
+
+
+def top_p_ratio(s_anc: float, s_max: float, s_min: float) -> float:
+    """Eq. 2: P = (s_max - s_anc) / (s_max - s_min) if s_anc in (s_min, s_max], else 0."""
+    if s_min < s_anc <= s_max:
+        return (s_max - s_anc) / (s_max - s_min)
+    return 0.0
+
+
+def middle_units(L_c: int, B: int, n_init: int, n_local: int) -> list[int]:
+    prot = set(protected_units(L_c, B, n_init, n_local))
+    return [m for m in range(-(-L_c // B)) if m not in prot]
+
+
+def top_p_per_head(u: np.ndarray, ctx_offsets, B: int, n_init: int, n_local: int,
+                   max_units=None, min_units=None) -> np.ndarray:
+    """P^(n)_doc-i for one layer (and batch element): [Hkv, D].  s_max / s_min are the scores of the
+    caller's max / min blocks (global unit ids [D], from the offline analysis of Appendix A.1) or,
+    when none are given, the largest / smallest middle-unit score.  A context without middle
+    units gets 0."""
+    u = np.asarray(u, dtype=F64)
+    nb, unit_off = unit_layout(ctx_offsets, B)
+    D = len(nb)
+    P = np.zeros((u.shape[0], D), dtype=F64)
+    for h in range(u.shape[0]):
+        for c in range(D):
+            L_c = int(ctx_offsets[c + 1]) - int(ctx_offsets[c])
+            mid = middle_units(L_c, B, n_init, n_local)
+            if not mid:
+                continue
+            vals = [float(u[h, unit_off[c] + m]) for m in mid]
+            s_max = float(u[h, int(max_units[c])]) if max_units is not None else max(vals)
+            s_min = float(u[h, int(min_units[c])]) if min_units is not None else min(vals)
+            P[h, c] = top_p_ratio(anchor_score(u[h], c, ctx_offsets, B, n_init, n_local), s_max, s_min)
+    return P
+
+
+def consolidate_top_p(P_layers: np.ndarray) -> np.ndarray:
+    """Eq. 3: P_doc-i = mean over the stable layers N* of P^(n)_doc-i.  P_layers: [|N*|, Hkv, D];
+    the paper has no head index, so the KV heads are averaged too: one ratio per document."""
+    P_layers = np.asarray(P_layers, dtype=F64)
+    D = P_layers.shape[-1]
+    out = np.zeros(D, dtype=F64)
+    for c in range(D):
+        tot = 0.0
+        for n in range(P_layers.shape[0]):
+            for h in range(P_layers.shape[1]):
+                tot += P_layers[n, h, c]
+        out[c] = tot / (P_layers.shape[0] * P_layers.shape[1])
+    return out
+
+
+def candidate_counts(P_doc: np.ndarray, ctx_offsets, B: int, n_init: int, n_local: int) -> list[int]:
+    """Top-P of a document: floor(P * number of middle units) middle units."""
+    out = []
+    for c, P in enumerate(P_doc):
+        L_c = int(ctx_offsets[c + 1]) - int(ctx_offsets[c])
+        n_mid = len(middle_units(L_c, B, n_init, n_local))
+        out.append(max(0, min(n_mid, int(np.floor(float(P) * n_mid + 1e-12)))))
+    return out
+
+
+def cross_context_select(u: np.ndarray, ctx_offsets, B: int, n_init: int, n_local: int, cand_counts):
+    """Section 3.2, last paragraph.  Per KV head: in every context the cand_counts[c] best middle
+    units are retrieved; their scores are min-max normalised inside their context
+    ((u - min) / (max - min) over that context's middle units; 0 if max == min); the retrieved
+    units of all contexts are compared and the best K = floor(total retrieved / D) are kept
+    (equal normalised scores: lower global unit id first).  Protected units are always kept.
+    Returns (sel [Hkv, S_u] ascending global unit ids, counts [Hkv, D] units kept per context)."""
+    u = np.asarray(u, dtype=F64)
+    Hkv = u.shape[0]
+    nb, unit_off = unit_layout(ctx_offsets, B)
+    D = len(nb)
+    C = int(sum(int(c) for c in cand_counts))
+    K = C // D
+    prot_all = []
+    for c in range(D):
+        L_c = int(ctx_offsets[c + 1]) - int(ctx_offsets[c])
+        prot_all.append([unit_off[c] + m for m in protected_units(L_c, B, n_init, n_local)])
+    S_u = sum(len(p) for p in prot_all) + K
+    sel = np.zeros((Hkv, S_u), dtype=np.int32)
+    counts = np.zeros((Hkv, D), dtype=np.int32)
+    for h in range(Hkv):
+        pool = []                                   # (normalised score, global unit id)
+        for c in range(D):
+            L_c = int(ctx_offsets[c + 1]) - int(ctx_offsets[c])
+            mid = middle_units(L_c, B, n_init, n_local)
+            if not mid or cand_counts[c] == 0:
+                continue
+            vals = {m: float(u[h, unit_off[c] + m]) for m in mid}
+            lo, hi = min(vals.values()), max(vals.values())
+            order = sorted(mid, key=lambda m: (-vals[m], m))[: int(cand_counts[c])]
+            for m in order:
+                v = (vals[m] - lo) / (hi - lo) if hi > lo else 0.0
+                pool.append((v, unit_off[c] + m))
+        chosen = sorted(pool, key=lambda t: (-t[0], t[1]))[:K]
+        kept = sorted([uid for _, uid in chosen] + [uid for p in prot_all for uid in p])
+        sel[h] = kept
+        for uid in kept:
+            c = 0
+            while not (unit_off[c] <= uid < unit_off[c + 1]):
+                c += 1
+            counts[h, c] += 1
+    return sel, counts

@@ -482,3 +482,102 @@ def test_sparsify_stage_shapes_and_counts():
     for h in range(2):
         counts = [int(((res["sel"][h] >= off[c]) & (res["sel"][h] < off[c + 1])).sum()) for c in range(3)]
         assert counts == [3, 4, 2]
+
+
+# ----------------------------------------------------------------------------- Eq. 2 / Eq. 3 / cross-context Top-K
+def test_eq2_hand_values_and_interval_ends():
+    assert O.top_p_ratio(s_anc=2.0, s_max=4.0, s_min=0.0) == 0.5
+    assert O.top_p_ratio(1.0, 4.0, 0.0) == 0.75                       # a low anchor lets more blocks through
+    assert O.top_p_ratio(4.0, 4.0, 0.0) == 0.0                        # s_anc = s_max: inside the interval, P = 0
+    assert O.top_p_ratio(0.0, 4.0, 0.0) == 0.0                        # s_anc = s_min: outside (open end)
+    assert O.top_p_ratio(5.0, 4.0, 0.0) == 0.0 and O.top_p_ratio(-1.0, 4.0, 0.0) == 0.0
+    assert O.top_p_ratio(1.0, 1.0, 1.0) == 0.0                        # degenerate: no division by zero
+    assert abs(O.top_p_ratio(1e-9, 1.0, 0.0) - 1.0) < 1e-8            # s_anc -> s_min+ : P -> 1
+
+
+def test_anchor_score_is_token_weighted_mean_of_protected_units():
+    ctx = [0, 22]                     # B = 4: units of 4,4,4,4,4,2 tokens; init = unit 0, local (last 4 tokens) = units 4,5
+    u = np.array([10.0, 1.0, 2.0, 3.0, 20.0, 40.0])
+    assert O.protected_units(22, 4, 4, 4) == [0, 4, 5]
+    assert O.anchor_score(u, 0, ctx, 4, 4, 4) == pytest.approx((10 * 4 + 20 * 4 + 40 * 2) / 10)
+    assert O.middle_units(22, 4, 4, 4) == [1, 2, 3]
+
+
+def test_top_p_per_head_default_and_caller_blocks_and_eq3():
+    ctx = [0, 24, 40]                 # B = 4, init 4, local 4 -> ctx0 units 0..5 (middle 1..4), ctx1 units 6..9 (middle 7,8)
+    u = np.array([[2.0, 5.0, 1.0, 3.0, 4.0, 2.0,   0.0, 9.0, 1.0, 0.0],
+                  [9.0, 5.0, 1.0, 3.0, 4.0, 9.0,   3.0, 2.0, 6.0, 3.0]])
+    P = O.top_p_per_head(u, ctx, 4, 4, 4)
+    # head 0 ctx 0: anc = 2, max 5, min 1 -> 3/4 ; ctx 1: anc 0 < min 1 -> 0
+    # head 1 ctx 0: anc 9 > max -> 0 ;           ctx 1: anc 3, max 6, min 2 -> 3/4
+    assert np.allclose(P, [[0.75, 0.0], [0.0, 0.75]])
+    P2 = O.top_p_per_head(u, ctx, 4, 4, 4, max_units=[4, 8], min_units=[3, 7])   # caller-supplied max/min blocks
+    # head 0 ctx 0: max 4, min 3, anc 2 -> not in (3,4] -> 0 ; ctx 1: max 1, min 9 -> empty interval -> 0
+    # head 1 ctx 0: 0 ; ctx 1: max 6, min 2, anc 3 -> 0.75
+    assert np.allclose(P2, [[0.0, 0.0], [0.0, 0.75]])
+    Pd = O.consolidate_top_p(np.stack([P, P2]))                      # Eq. 3 over two "stable layers" (and the heads)
+    assert np.allclose(Pd, [0.75 / 4, (0.75 + 0.75) / 4])
+    assert O.candidate_counts([0.74, 0.5, 1.0, 0.0], [0, 24, 40, 64, 88], 4, 4, 4) == [2, 1, 4, 0]
+
+
+def _cross_brute(u_row, ctx, B, n_init, n_local, cand):
+    """Independent route with numpy argsort on a (score, id) structured key."""
+    nb, off = O.unit_layout(ctx, B)
+    D = len(nb)
+    pool_v, pool_id, prot = [], [], []
+    for c in range(D):
+        L_c = ctx[c + 1] - ctx[c]
+        pr = O.protected_units(L_c, B, n_init, n_local)
+        prot += [off[c] + m for m in pr]
+        mid = np.array([m for m in range(nb[c]) if m not in set(pr)], dtype=int)
+        if len(mid) == 0 or cand[c] == 0:
+            continue
+        vals = u_row[off[c] + mid]
+        order = np.lexsort((mid, -vals))[: cand[c]]
+        lo, hi = vals.min(), vals.max()
+        pool_v += list(((vals[order] - lo) / (hi - lo)) if hi > lo else np.zeros(len(order)))
+        pool_id += list(off[c] + mid[order])
+    K = sum(cand) // D
+    pool_v, pool_id = np.array(pool_v), np.array(pool_id, dtype=int)
+    pick = np.lexsort((pool_id, -pool_v))[:K] if len(pool_v) else []
+    return sorted(prot + [int(pool_id[i]) for i in pick])
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_cross_context_select_against_brute_force(seed):
+    r = np.random.default_rng(100 + seed)
+    B = [1, 4, 8, 2, 1][seed]
+    lens = [int(x) for x in r.integers(6 * B, 20 * B, size=4)]
+    ctx = [0] + [int(x) for x in np.cumsum(lens)]
+    nb, off = O.unit_layout(ctx, B)
+    u = r.integers(0, 7, size=(2, off[-1])).astype(float) if seed % 2 else r.normal(size=(2, off[-1]))
+    cand = [int(r.integers(0, len(O.middle_units(lens[c], B, B, 2 * B)) + 1)) for c in range(4)]
+    sel, counts = O.cross_context_select(u, ctx, B, B, 2 * B, cand)
+    K = sum(cand) // 4
+    n_prot = sum(len(O.protected_units(n, B, B, 2 * B)) for n in lens)
+    assert sel.shape == (2, n_prot + K)
+    for h in range(2):
+        assert list(sel[h]) == _cross_brute(u[h], ctx, B, B, 2 * B, cand)
+        assert counts[h].sum() == n_prot + K and np.all(np.diff(sel[h]) > 0)
+
+
+def test_cross_context_select_properties():
+    r = np.random.default_rng(7)
+    ctx = [0, 30, 70, 95]
+    u = r.normal(size=(1, 95))
+    cand = [6, 9, 4]
+    sel, counts = O.cross_context_select(u, ctx, 1, 2, 3, cand)
+    # min-max normalisation: an affine map (a > 0) of one context's scores changes nothing
+    u2 = u.copy(); u2[0, 30:70] = 3.5 * u2[0, 30:70] - 11.0
+    sel2, _ = O.cross_context_select(u2, ctx, 1, 2, 3, cand)
+    assert np.array_equal(sel, sel2)
+    # one context: K = all its candidates, i.e. the fixed-budget selection with k = protected + candidates
+    s1, c1 = O.cross_context_select(u[:, :30], [0, 30], 1, 2, 3, [6])
+    assert np.array_equal(s1, O.select_units(u[:, :30], [0, 30], 1, 2, 3, [5 + 6]))
+    # nothing retrieved: only the protected units survive (the "no selection" ablation)
+    s0, c0 = O.cross_context_select(u, ctx, 1, 2, 3, [0, 0, 0])
+    assert list(s0[0]) == [0, 1, 27, 28, 29, 30, 31, 67, 68, 69, 70, 71, 92, 93, 94]
+    # the best unit of a context normalises to 1 and always wins a place when K >= number of contexts with candidates
+    for c in range(3):
+        lo, hi = ctx[c] + 2, ctx[c + 1] - 3
+        assert (lo + int(np.argmax(u[0, lo:hi]))) in sel[0]
