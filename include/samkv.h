@@ -179,6 +179,55 @@ samkv_status_t samkv_attn(samkv_handle_t h, const samkv_shape_t* shape, int32_t 
                           int32_t cache_capacity, int32_t* cache_len, const void* Q, int32_t T_q, const void* Kq,
                           const void* Vq, float scale, void* O, float* lse, void* stream);
 
+/* ---- the paper's dynamic selection: Top-P per document, then Top-K across documents --------------- */
+
+#define SAMKV_MAX_STAR_LAYERS 64
+
+/* Dynamic Top-P (Sec. 3.2, Eq. 2; consolidated over the stable layers N*, Eq. 3).  Per stable layer n, batch
+ * element, KV head and document i:
+ *   s_anc = score of the anchor = token-weighted mean of the protected (initial + local) units' scores
+ *   s_max, s_min = scores of the document's max / min blocks (max_units / min_units: device int32 [L, Bt, D],
+ *                  global unit ids from the offline attention analysis of App. A.1), or, when the pointer is
+ *                  NULL, the largest / smallest middle-unit score
+ *   P^(n) = (s_max - s_anc) / (s_max - s_min)  if s_anc in (s_min, s_max],  else 0      (also 0 without middle units)
+ * P_out[b, i] = mean over n in N* and over the KV heads (the paper has no head index).
+ *   scores      fp32 [L, Bt, Hkv, U_tot] from samkv_score
+ *   star_layers host [n_star], 1 <= n_star <= SAMKV_MAX_STAR_LAYERS, layer indices in [0, L)
+ *   P_out       device fp32 [Bt, D] */
+samkv_status_t samkv_topp(samkv_handle_t h, const samkv_shape_t* shape, const float* scores, const int32_t* star_layers,
+                          int32_t n_star, const int32_t* max_units, const int32_t* min_units, float* P_out,
+                          void* stream);
+
+/* Host helper: from one request's ratios P (host [D]) the number of middle units retrieved per document,
+ * cand[i] = floor(P[i] * middle units of i), the cross-context K = floor(sum cand / D), the length
+ * S_u = protected units + K of every selection list, and the kept-token count S.  Outputs may be NULL. */
+samkv_status_t samkv_topp_plan(const samkv_shape_t* shape, const float* P, int32_t* cand_out, int32_t* K_out,
+                               int32_t* S_u_out, int32_t* kept_tokens_out);
+
+/* Cross-context Top-K (Sec. 3.2, last paragraph).  Per (layer, batch, KV head): document i retrieves its cand[i]
+ * best middle units (ties: lower index); their scores are min-max normalised inside the document over its
+ * middle units ((u - min) / (max - min), 0 if max == min); the K = floor(sum cand / D) best of all retrieved
+ * units are kept (equal normalised scores: lower global unit id), together with every protected unit.
+ *   cand       host [D]
+ *   scratch    device, 16-byte aligned, at least samkv_select_cross_scratch_bytes(shape, cand) bytes, owned by
+ *              the caller and free again when the call's work on `stream` has finished; it holds one
+ *              (key, unit id) pair per retrieved unit.  With cand == NULL the size helper returns the bound
+ *              for any cand (every middle unit retrieved).
+ *   sel_out    int32 [L, Bt, Hkv, S_u] ascending global unit ids, S_u = protected units + K
+ *   counts_out int32 [L, Bt, Hkv, D] optional: units kept per document (they differ from head to head)
+ * SAMKV_ERR_BUDGET if some cand[i] exceeds the document's middle units; SAMKV_ERR_WORKSPACE if scratch is short. */
+size_t samkv_select_cross_scratch_bytes(const samkv_shape_t* shape, const int32_t* cand);
+samkv_status_t samkv_select_cross(samkv_handle_t h, const samkv_shape_t* shape, const float* scores,
+                                  const int32_t* cand, void* scratch, size_t scratch_bytes, int32_t* sel_out,
+                                  int32_t* counts_out, void* stream);
+
+/* Compaction for a selection list whose split between documents is free (as samkv_select_cross writes it):
+ * sel int32 [L, Bt, Hkv, S_u] ascending global unit ids that contain every short tail unit.  Otherwise as
+ * samkv_compact (V may be pinned host memory; cache_len set to the kept-token count; optional inv_map). */
+samkv_status_t samkv_compact_units(samkv_handle_t h, const samkv_shape_t* shape, const void* K, const void* V,
+                                   const int32_t* sel, int32_t S_u, void* Kc, void* Vc, int32_t cache_capacity,
+                                   int32_t* cache_len, int32_t* inv_map, void* stream);
+
 /* ---- scoring without any allocation ------------------------------------------------------ */
 
 /* (No counterpart in the paper: this entry point exists for deployment reasons only.)

@@ -25,7 +25,8 @@ STATUS_NAMES = {0: "SAMKV_OK", 1: "SAMKV_ERR_INVALID_ARG", 2: "SAMKV_ERR_UNSUPPO
 
 EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll_status", "samkv_status_string",
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
-           "samkv_attn", "samkv_score_static"]
+           "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
+           "samkv_select_cross_scratch_bytes", "samkv_compact_units"]
 
 
 class SamkvError(RuntimeError):
@@ -69,6 +70,13 @@ def lib() -> ctypes.CDLL:
     L.samkv_update.argtypes = [vp, shp, vp, vp, i32, vp, vp, i32, vp, vp, i32, vp]
     L.samkv_attn.argtypes = [vp, shp, i32, vp, vp, i32, vp, vp, i32, vp, vp, f32, vp, vp, vp]
     L.samkv_score_static.argtypes = [shp, vp, vp, i32, vp, i32, i32, vp, vp]
+    f32p = ctypes.POINTER(ctypes.c_float)
+    L.samkv_topp.argtypes = [vp, shp, vp, i32p, i32, vp, vp, vp, vp]
+    L.samkv_topp_plan.argtypes = [shp, f32p, i32p, i32p, i32p, i32p]
+    L.samkv_select_cross.argtypes = [vp, shp, vp, i32p, vp, ctypes.c_size_t, vp, vp, vp]
+    L.samkv_select_cross_scratch_bytes.argtypes = [shp, i32p]
+    L.samkv_select_cross_scratch_bytes.restype = ctypes.c_size_t
+    L.samkv_compact_units.argtypes = [vp, shp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("samkv_status_string", "samkv_workspace_bytes"):
             getattr(L, name).restype = ctypes.c_int
@@ -221,3 +229,38 @@ def samkv_score_static(shape: Shape, K, Q, T_q: int, Qloc, T_loc: int, use_bias:
     the scratch is a fixed 1 MiB array inside the library.  Calls sharing a GPU must not overlap."""
     _check(lib().samkv_score_static(shape.ref(), _ptr(K), _ptr(Q), T_q, _ptr(Qloc), T_loc, int(use_bias),
                                     _ptr(scores_out), _stream()), "samkv_score_static")
+
+
+# ------------------------------------------------------------------ dynamic selection (Eq. 2, Eq. 3, cross-context Top-K)
+def samkv_topp(handle: Handle, shape: Shape, scores, star_layers: Sequence[int], max_units, min_units, P_out):
+    _check(lib().samkv_topp(handle.h, shape.ref(), _ptr(scores), _i32_array(star_layers), len(star_layers),
+                            _ptr(max_units), _ptr(min_units), _ptr(P_out), _stream()), "samkv_topp")
+
+
+def samkv_topp_plan(shape: Shape, P: Sequence[float]):
+    """Returns (cand per document, K, S_u, kept tokens S) for one request's Top-P ratios."""
+    arr = (ctypes.c_float * len(P))(*[float(x) for x in P])
+    cand = (ctypes.c_int32 * shape.n_ctx)()
+    K, S_u, S = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().samkv_topp_plan(shape.ref(), arr, cand, ctypes.byref(K), ctypes.byref(S_u), ctypes.byref(S)),
+           "samkv_topp_plan")
+    return list(cand), K.value, S_u.value, S.value
+
+
+def samkv_select_cross_scratch_bytes(shape: Shape, cand: Optional[Sequence[int]] = None) -> int:
+    """Bytes of scratch samkv_select_cross needs for these candidate counts (None: the bound for any counts)."""
+    return int(lib().samkv_select_cross_scratch_bytes(shape.ref(), None if cand is None else _i32_array(cand)))
+
+
+def samkv_select_cross(handle: Handle, shape: Shape, scores, cand: Sequence[int], scratch, sel_out, counts_out=None):
+    """scratch: a device tensor of at least samkv_select_cross_scratch_bytes(shape) bytes."""
+    _check(lib().samkv_select_cross(handle.h, shape.ref(), _ptr(scores), _i32_array(cand), _ptr(scratch),
+                                    scratch.numel() * scratch.element_size(), _ptr(sel_out), _ptr(counts_out),
+                                    _stream()), "samkv_select_cross")
+
+
+def samkv_compact_units(handle: Handle, shape: Shape, K, V, sel, S_u: int, Kc, Vc, cache_capacity: int, cache_len,
+                        inv_map=None):
+    _check(lib().samkv_compact_units(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(sel), S_u,
+                                     _ptr(Kc), _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()),
+           "samkv_compact_units")

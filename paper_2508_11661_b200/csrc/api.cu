@@ -336,4 +336,115 @@ samkv_status_t samkv_attn(samkv_handle_t handle, const samkv_shape_t* shape, int
                                h->workspace + ws_off, plan, h->d_status, static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_topp(samkv_handle_t handle, const samkv_shape_t* shape, const float* scores,
+                          const int32_t* star_layers, int32_t n_star, const int32_t* max_units,
+                          const int32_t* min_units, float* P_out, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (scores == nullptr || P_out == nullptr || star_layers == nullptr) return SAMKV_ERR_INVALID_ARG;
+  if (n_star < 1 || n_star > SAMKV_MAX_STAR_LAYERS) return SAMKV_ERR_INVALID_ARG;
+  for (int i = 0; i < n_star; ++i)
+    if (star_layers[i] < 0 || star_layers[i] >= shape->n_layers) return SAMKV_ERR_INVALID_ARG;
+  return from_cuda(launch_topp(*shape, lo.ct, lo.n_init_units, lo.first_local_unit, scores, star_layers, n_star,
+                               max_units, min_units, P_out, static_cast<cudaStream_t>(stream)));
+}
+
+// cand, K, S_u, kept tokens of the cross-context selection; shared by the plan helper and the two calls below
+static samkv_status_t cross_plan(const samkv_shape_t* shape, const Layout& lo, const int32_t* cand, int* K, int* S_u,
+                                 int* S) {
+  long long total = 0, n_prot = 0, deficit = 0;
+  for (int c = 0; c < shape->n_ctx; ++c) {
+    const int n_mid = lo.nb[c] - lo.n_prot[c];
+    if (cand[c] < 0 || cand[c] > n_mid) return SAMKV_ERR_BUDGET;
+    total += cand[c];
+    n_prot += lo.n_prot[c];
+    deficit += shape->block_size - lo.tail[c];
+  }
+  *K = (int)(total / shape->n_ctx);
+  *S_u = (int)(n_prot + *K);
+  *S = (int)((long long)*S_u * shape->block_size - deficit);
+  return SAMKV_OK;
+}
+
+samkv_status_t samkv_topp_plan(const samkv_shape_t* shape, const float* P, int32_t* cand_out, int32_t* K_out,
+                               int32_t* S_u_out, int32_t* kept_tokens_out) {
+  Layout lo;
+  samkv_status_t st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (P == nullptr) return SAMKV_ERR_INVALID_ARG;
+  int32_t cand[SAMKV_MAX_CTX];
+  for (int c = 0; c < shape->n_ctx; ++c) {
+    if (!(P[c] >= 0.0f && P[c] <= 1.0f)) return SAMKV_ERR_INVALID_ARG;       // also refuses NaN
+    const int n_mid = lo.nb[c] - lo.n_prot[c];
+    int k = (int)((double)P[c] * n_mid + 1e-12);
+    if (k > n_mid) k = n_mid;
+    cand[c] = k;
+    if (cand_out != nullptr) cand_out[c] = k;
+  }
+  int K = 0, S_u = 0, S = 0;
+  st = cross_plan(shape, lo, cand, &K, &S_u, &S);
+  if (st != SAMKV_OK) return st;
+  if (K_out != nullptr) *K_out = K;
+  if (S_u_out != nullptr) *S_u_out = S_u;
+  if (kept_tokens_out != nullptr) *kept_tokens_out = S;
+  return SAMKV_OK;
+}
+
+size_t samkv_select_cross_scratch_bytes(const samkv_shape_t* shape, const int32_t* cand) {
+  Layout lo;
+  if (make_layout(shape, &lo) != SAMKV_OK) return 0;
+  size_t per_slab = 0;                                  // one (key, unit id) pair per retrieved unit
+  for (int c = 0; c < shape->n_ctx; ++c) {
+    const int n_mid = lo.nb[c] - lo.n_prot[c];
+    per_slab += (size_t)(cand == nullptr ? n_mid : (cand[c] < 0 ? 0 : (cand[c] < n_mid ? cand[c] : n_mid)));
+  }
+  const size_t bytes = (size_t)shape->n_layers * shape->batch * shape->n_kv_heads * per_slab * 8;
+  return bytes < 16 ? 16 : bytes;
+}
+
+samkv_status_t samkv_select_cross(samkv_handle_t handle, const samkv_shape_t* shape, const float* scores,
+                                  const int32_t* cand, void* scratch, size_t scratch_bytes, int32_t* sel_out,
+                                  int32_t* counts_out, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (scores == nullptr || cand == nullptr || sel_out == nullptr) return SAMKV_ERR_INVALID_ARG;
+  int K = 0, S_u = 0, S = 0;
+  st = cross_plan(shape, lo, cand, &K, &S_u, &S);
+  if (st != SAMKV_OK) return st;
+  if (scratch == nullptr || !aligned16(scratch)) return SAMKV_ERR_INVALID_ARG;
+  if (scratch_bytes < samkv_select_cross_scratch_bytes(shape, cand)) return SAMKV_ERR_WORKSPACE;
+  return from_cuda(launch_select_cross(*shape, lo.ct, lo.n_init_units, lo.first_local_unit, scores, cand, K, S_u, scratch,
+                                       sel_out, counts_out, h->max_smem_optin, static_cast<cudaStream_t>(stream)));
+}
+
+samkv_status_t samkv_compact_units(samkv_handle_t handle, const samkv_shape_t* shape, const void* K, const void* V,
+                                   const int32_t* sel_in, int32_t S_u, void* Kc, void* Vc, int32_t cache_capacity,
+                                   int32_t* cache_len, int32_t* inv_map, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (K == nullptr || V == nullptr || sel_in == nullptr || Kc == nullptr || Vc == nullptr || cache_len == nullptr)
+    return SAMKV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc)) return SAMKV_ERR_INVALID_ARG;
+  long long n_prot = 0, deficit = 0;
+  for (int c = 0; c < shape->n_ctx; ++c) { n_prot += lo.n_prot[c]; deficit += shape->block_size - lo.tail[c]; }
+  if (S_u < n_prot || S_u > lo.U_tot) return SAMKV_ERR_BUDGET;
+  const int S = (int)((long long)S_u * shape->block_size - deficit);
+  if (cache_capacity < S) return SAMKV_ERR_CAPACITY;
+  return from_cuda(launch_compact_units(*shape, lo.ct, lo.n_init_units, lo.first_local_unit, K, V, sel_in, S_u, S, Kc, Vc,
+                                        cache_capacity, cache_len, inv_map, h->d_status,
+                                        static_cast<cudaStream_t>(stream)));
+}
+
 }  // extern "C"

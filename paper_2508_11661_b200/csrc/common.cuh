@@ -49,6 +49,17 @@ cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc,
                           const int32_t* tok_ids, int R, const void* Knew, const void* Vnew, int mode,
                           cudaStream_t stream);
 
+cudaError_t launch_topp(const samkv_shape_t& s, const CtxTable& ct, const int* n_init_units, const int* first_local_unit,
+                        const float* scores, const int32_t* star_layers, int n_star, const int32_t* max_units,
+                        const int32_t* min_units, float* P_out, cudaStream_t stream);
+cudaError_t launch_select_cross(const samkv_shape_t& s, const CtxTable& ct, const int* n_init_units,
+                                const int* first_local_unit, const float* scores, const int32_t* cand, int K, int S_u,
+                                void* scratch, int32_t* sel, int32_t* counts, int max_smem_optin, cudaStream_t stream);
+cudaError_t launch_compact_units(const samkv_shape_t& s, const CtxTable& ct, const int* n_init_units,
+                                 const int* first_local_unit, const void* K, const void* V, const int32_t* sel, int S_u,
+                                 int S, void* Kc, void* Vc, int capacity, int32_t* cache_len, int32_t* inv_map,
+                                 int* d_status, cudaStream_t stream);
+
 struct AttnPlan {
   int n_splits;        // KV splits per (batch, kv head, row tile)
   int rows_per_cta;    // packed query rows (T_q * G) per CTA

@@ -67,6 +67,31 @@ def test_budget_and_layout_match_oracle(seed):
         assert S == len(O.units_to_tokens(sel[0], off, Bsz))
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_topp_plan_matches_oracle(seed):
+    """Candidate counts, K, list length and kept tokens of the dynamic selection (host arithmetic only)."""
+    r = np.random.default_rng(100 + seed)
+    Bsz = int(2 ** r.integers(0, 7))
+    n_init = Bsz * int(r.integers(0, 3))
+    n_local = Bsz * int(r.integers(1, 4))
+    lens = [int(x) for x in r.integers(1, 2000, size=int(r.integers(1, 9)))]
+    off = [0] + list(np.cumsum(lens))
+    shape = B.Shape(1, 1, 8, 2, 128, off, Bsz, n_init, n_local, "bf16")
+    _, U_tot, _ = B.samkv_layout(shape)
+    for trial in range(4):
+        P = r.random(len(lens)).astype(np.float32)
+        if trial == 0:
+            P[:] = 0.0
+        if trial == 1:
+            P[:] = 1.0
+        cand, K, S_u, S = B.samkv_topp_plan(shape, [float(x) for x in P])
+        assert cand == O.candidate_counts(P.astype(np.float64), off, Bsz, n_init, n_local)
+        u = r.normal(size=(2, U_tot))
+        sel, counts = O.cross_context_select(u, off, Bsz, n_init, n_local, cand)
+        assert K == sum(cand) // len(lens) and S_u == sel.shape[1]
+        assert S == len(O.units_to_tokens(sel[0], off, Bsz)) == len(O.units_to_tokens(sel[1], off, Bsz))
+
+
 def test_bad_shapes_are_refused_on_the_host():
     ok = dict(n_layers=1, batch=1, n_q_heads=8, n_kv_heads=2, head_dim=128, ctx_offsets=[0, 100, 300], block_size=1,
               n_init=4, n_local=8, dtype="bf16")
