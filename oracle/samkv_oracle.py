@@ -20,7 +20,10 @@ context c on the concatenated token axis, k_units[c] units kept in context c.
 
 Pins (tests/test_oracle_pins.py): closed forms of Eq. 1 and Eq. 4, linearity of the
 block-mean score, brute-force selection, bit-exact gather, softmax invariants, the
-100 %-budget == full-attention invariant, and torch's fp64 scaled_dot_product_attention.
+100 %-budget == full-attention invariant, torch's fp64 scaled_dot_product_attention, hand
+values / brute force / invariances for Eq. 2-3 and the cross-context Top-K, and for the
+cross-layer alignment the four token cases of the paper's recomputation figure plus a
+layer-by-layer simulation that checks the plan is sufficient and minimal.
 The paper prints no worked numerical example of Eq. 1-4, so parity with the paper's
 own numbers is unpinned; every function below is pinned by mathematics instead.
 """
@@ -544,3 +547,63 @@ def cross_context_select(u: np.ndarray, ctx_offsets, B: int, n_init: int, n_loca
                 c += 1
             counts[h, c] += 1
     return sel, counts
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.3 "Recomputation": blank-block alignment across layers and the two rules
+# --------------------------------------------------------------------------------------
+FLAG_KEPT = 1        # some KV head of this layer keeps the token (not a blank position)
+FLAG_RECOMPUTE = 2   # the token's K/V of this layer are recomputed (rule 2, "when necessary")
+FLAG_OUTPUT = 4      # this layer must also produce the token's output (rule 1: a higher layer recomputes it)
+FLAG_PAD_REUSE = 8   # blank here, yet on the forward path: its prefilled K/V entry is used for the output
+
+
+def align_layers(inv_map: np.ndarray, tok_ids: np.ndarray):
+    """Pad -> merge -> recompute plan -> (the caller removes the padding again).
+
+    inv_map [L, Hkv, L_tot]: slot of token t in the compact cache of (layer, head), -1 = blank.
+    tok_ids [L, R]: tokens whose K/V should be recomputed at each layer (-1 = unused entry).
+
+    A token is a blank position of layer n when no head of that layer keeps it.  Laying every
+    layer over the union of all layers' kept tokens (the merged axis) aligns them; the blanks
+    are the padding.  For layer n and token t:
+      recompute  t is listed for layer n and layer n keeps it (a listed token that is blank at
+                 layer n has no cache entry to refresh);
+      output     some layer m > n recomputes t: computing t's K/V at layer m needs t's hidden
+                 state, hence the outputs of every layer below m (rule 1);
+      pad_reuse  output is needed, t is not recomputed here and is blank here: the forward pass
+                 takes t's prefilled K/V entry (rule 2 reuses what exists).
+    Returns (flags [L, L_tot] uint8, merged token ids ascending, per-layer ascending lists of
+    the tokens that enter the layer's forward pass = recompute or output)."""
+    inv_map = np.asarray(inv_map)
+    tok_ids = np.asarray(tok_ids)
+    L, Hkv, L_tot = inv_map.shape
+    flags = np.zeros((L, L_tot), dtype=np.uint8)
+    merged = []
+    for t in range(L_tot):
+        on_axis = False
+        for n in range(L):
+            kept = any(inv_map[n, h, t] >= 0 for h in range(Hkv))
+            on_axis = on_axis or kept
+            listed = any(int(x) == t for x in tok_ids[n])
+            rec = listed and kept
+            f = 0
+            if kept:
+                f |= FLAG_KEPT
+            if rec:
+                f |= FLAG_RECOMPUTE
+            flags[n, t] = f
+        if on_axis:
+            merged.append(t)
+    for t in range(L_tot):
+        for n in range(L):
+            higher = any(flags[m, t] & FLAG_RECOMPUTE for m in range(n + 1, L))
+            if higher:
+                flags[n, t] |= FLAG_OUTPUT
+                if not (flags[n, t] & FLAG_RECOMPUTE) and not (flags[n, t] & FLAG_KEPT):
+                    flags[n, t] |= FLAG_PAD_REUSE
+    run = []
+    for n in range(L):
+        run.append(np.asarray([t for t in range(L_tot) if flags[n, t] & (FLAG_RECOMPUTE | FLAG_OUTPUT)],
+                              dtype=np.int64))
+    return flags, np.asarray(merged, dtype=np.int64), run

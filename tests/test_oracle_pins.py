@@ -581,3 +581,63 @@ def test_cross_context_select_properties():
     for c in range(3):
         lo, hi = ctx[c] + 2, ctx[c + 1] - 3
         assert (lo + int(np.argmax(u[0, lo:hi]))) in sel[0]
+
+
+# ------------------------------------------------------------------------------------------
+# Section 3.3: blank-block alignment and the two recomputation rules
+# ------------------------------------------------------------------------------------------
+def test_align_layers_the_four_cases_of_the_recomputation_figure():
+    """Two layers, one head.  Tokens: 0 lower layer recomputed / upper not; 1 neither; 2 upper recomputed /
+    lower not, and blank in the lower layer; 3 both; 4 blank everywhere but listed; 5 upper recomputed, lower
+    kept and not recomputed.  Expected flags follow the paper's discussion of its examples 1-4."""
+    K, R, Out, Pad = O.FLAG_KEPT, O.FLAG_RECOMPUTE, O.FLAG_OUTPUT, O.FLAG_PAD_REUSE
+    inv = np.full((2, 1, 6), -1, dtype=np.int32)
+    inv[0, 0, [0, 1, 3, 5]] = [0, 1, 2, 3]          # lower layer keeps 0, 1, 3, 5 (2 and 4 are blanks)
+    inv[1, 0, [0, 1, 2, 3, 5]] = [0, 1, 2, 3, 4]    # upper layer keeps 0, 1, 2, 3, 5
+    tok = np.array([[0, 3, 4, -1], [2, 3, 5, -1]])
+    flags, merged, run = O.align_layers(inv, tok)
+    assert flags[:, 0].tolist() == [K | R, K]                 # (1) K/V refreshed below, no output needed
+    assert flags[:, 1].tolist() == [K, K]                     # (2) nothing to do
+    assert flags[:, 2].tolist() == [Out | Pad, K | R]         # (3) output below from the prefilled entry
+    assert flags[:, 3].tolist() == [K | R | Out, K | R]       # (4)
+    assert flags[:, 4].tolist() == [0, 0]                     # listed but blank: nothing to refresh
+    assert flags[:, 5].tolist() == [K | Out, K | R]           # output below, K/V reused from the compact cache
+    assert merged.tolist() == [0, 1, 2, 3, 5]
+    assert run[0].tolist() == [0, 2, 3, 5] and run[1].tolist() == [2, 3, 5]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_align_layers_plan_is_sufficient_and_minimal(seed):
+    """Demand analysis written the other way round: the hidden state of t is needed at the input of layer n iff
+    layer n recomputes t or the input of layer n+1 needs it.  The plan's forward lists must be exactly these
+    sets, and each layer's outputs exactly the next layer's inputs."""
+    r = np.random.default_rng(seed)
+    L, Hkv, T, R = int(r.integers(1, 7)), int(r.integers(1, 4)), 60, 9
+    inv = np.where(r.random((L, Hkv, T)) < 0.35, 1, -1).astype(np.int32)
+    tok = np.stack([r.permutation(T)[:R] for _ in range(L)])
+    tok[r.random(tok.shape) < 0.2] = -1
+    flags, merged, run = O.align_layers(inv, tok)
+    kept = (inv >= 0).any(axis=1)                                            # [L, T]
+    need = [set() for _ in range(L + 1)]
+    for n in reversed(range(L)):
+        rec_n = {int(t) for t in tok[n] if t >= 0 and kept[n, t]}
+        need[n] = rec_n | need[n + 1]
+        assert {t for t in range(T) if flags[n, t] & O.FLAG_RECOMPUTE} == rec_n
+    for n in range(L):
+        assert set(run[n].tolist()) == need[n]
+        assert {t for t in range(T) if flags[n, t] & O.FLAG_OUTPUT} == need[n + 1]
+        assert np.all(np.diff(run[n]) > 0)
+    assert not (flags[L - 1] & O.FLAG_OUTPUT).any()
+    assert merged.tolist() == [t for t in range(T) if kept[:, t].any()]
+    pad = (flags & O.FLAG_PAD_REUSE) != 0
+    assert np.array_equal(pad, ((flags & O.FLAG_OUTPUT) != 0) & ~kept & ((flags & O.FLAG_RECOMPUTE) == 0))
+    assert np.array_equal((flags & O.FLAG_KEPT) != 0, kept)
+
+
+def test_align_layers_without_recomputation_only_marks_kept_tokens():
+    inv = np.full((3, 2, 10), -1, dtype=np.int32)
+    inv[0, 0, 2] = 0
+    inv[2, 1, 7] = 0                                       # kept by one head only still counts as kept
+    flags, merged, run = O.align_layers(inv, np.full((3, 4), -1))
+    assert flags.sum() == 2 and flags[0, 2] == O.FLAG_KEPT and flags[2, 7] == O.FLAG_KEPT
+    assert merged.tolist() == [2, 7] and all(len(x) == 0 for x in run)
