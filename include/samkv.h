@@ -228,6 +228,32 @@ samkv_status_t samkv_compact_units(samkv_handle_t h, const samkv_shape_t* shape,
                                    const int32_t* sel, int32_t S_u, void* Kc, void* Vc, int32_t cache_capacity,
                                    int32_t* cache_len, int32_t* inv_map, void* stream);
 
+/* ---- cross-layer alignment of the sparse caches (Sec. 3.3 "Recomputation") ------------------------ */
+
+#define SAMKV_FLAG_KEPT 1       /* some KV head of the layer keeps the token (not a blank position) */
+#define SAMKV_FLAG_RECOMPUTE 2  /* K/V of the token are recomputed at this layer (rule 2) */
+#define SAMKV_FLAG_OUTPUT 4     /* the layer must produce the token's output: a higher layer recomputes it (rule 1) */
+#define SAMKV_FLAG_PAD_REUSE 8  /* blank here but on the forward path: the token's prefilled K/V entry is used */
+
+/* Pad -> merge -> recompute plan.  Layers (and heads) keep different tokens; laying every layer over the union
+ * of all layers' kept tokens aligns them, with blanks where a layer keeps nothing.  Per (layer n, batch b, token t):
+ *   KEPT       inv_map[n,b,h,t] >= 0 for some head h
+ *   RECOMPUTE  t is in tok_ids[n] and KEPT (a listed token that is blank at layer n has no entry to refresh)
+ *   OUTPUT     RECOMPUTE holds for t at some layer m > n (its K/V there need the outputs of all layers below)
+ *   PAD_REUSE  OUTPUT and not RECOMPUTE and not KEPT
+ *   inv_map     int32 [L, Bt, Hkv, L_tot] as written by samkv_compact / samkv_compact_units
+ *   tok_ids     int32 [L, R] (device) recompute lists as for samkv_update, -1 = unused entry; R may be 0
+ *   flags_out   uint8 [L, Bt, L_tot]
+ *   merged_ids  int32 [Bt, L_tot]: the merged axis, ascending token ids kept by any layer, then -1
+ *   merged_len  int32 [Bt]
+ *   run_ids     int32 [L, Bt, run_capacity]: ascending tokens with RECOMPUTE or OUTPUT (the layer's forward pass),
+ *               then -1; run_len int32 [L, Bt] always holds the full count
+ * A list longer than run_capacity is truncated and recorded as a device check (samkv_poll_status); so is a token
+ * id >= L_tot.  The caller removes the padding again by writing results through inv_map (samkv_update). */
+samkv_status_t samkv_align(samkv_handle_t h, const samkv_shape_t* shape, const int32_t* inv_map, const int32_t* tok_ids,
+                           int32_t R, uint8_t* flags_out, int32_t* merged_ids, int32_t* merged_len, int32_t* run_ids,
+                           int32_t run_capacity, int32_t* run_len, void* stream);
+
 /* ---- scoring without any allocation ------------------------------------------------------ */
 
 /* (No counterpart in the paper: this entry point exists for deployment reasons only.)

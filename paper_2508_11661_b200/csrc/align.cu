@@ -1,0 +1,116 @@
+// Cross-layer alignment of the sparse caches (Sec. 3.3): every layer is laid over the union of all layers' kept
+// tokens, positions a layer does not keep are blanks, and the two recomputation rules decide per (layer, token)
+// whether K/V are recomputed, whether the layer's output is needed, and whether a blank position feeds the
+// forward pass from its prefilled entry.  Pure integer work on inv_map and the recompute lists.
+#include "common.cuh"
+
+namespace samkv {
+
+constexpr int kAlignThreads = 256;
+constexpr uint8_t kFlagKept = 1, kFlagRecompute = 2, kFlagOutput = 4, kFlagPadReuse = 8;
+
+// flags[n, b, t] = "listed for recomputation at layer n" (tentative: the layer must also keep the token).
+__global__ void __launch_bounds__(kAlignThreads)
+align_mark_kernel(const int32_t* __restrict__ tok_ids, uint8_t* __restrict__ flags, int L, int Bt, int R, int L_tot,
+                  int* __restrict__ d_status) {
+  const int i = blockIdx.x * kAlignThreads + threadIdx.x;
+  if (i >= L * R) return;
+  const int n = i / R;
+  const int t = tok_ids[i];
+  if (t < 0) return;
+  if (t >= L_tot) {
+    atomicMax(d_status, (int)CHECK_SEL_RANGE);
+    return;
+  }
+  for (int b = 0; b < Bt; ++b) flags[((size_t)n * Bt + b) * L_tot + t] = kFlagRecompute;
+}
+
+// One thread per (batch element, token), layers from the top down: rule 1 propagates "recomputed above".
+__global__ void __launch_bounds__(kAlignThreads)
+align_flags_kernel(const int32_t* __restrict__ inv_map, uint8_t* __restrict__ flags, int L, int Bt, int Hkv, int L_tot) {
+  const int t = blockIdx.x * kAlignThreads + threadIdx.x;
+  const int b = blockIdx.y;
+  if (t >= L_tot) return;
+  bool above = false;                                           // some higher layer recomputes the token
+  for (int n = L - 1; n >= 0; --n) {
+    bool kept = false;
+    const int32_t* row = inv_map + (((size_t)n * Bt + b) * Hkv) * L_tot + t;
+    for (int h = 0; h < Hkv; ++h) kept = kept || (row[(size_t)h * L_tot] >= 0);
+    uint8_t* f = flags + ((size_t)n * Bt + b) * L_tot + t;
+    const bool rec = (*f != 0) && kept;
+    uint8_t v = 0;
+    if (kept) v |= kFlagKept;
+    if (rec) v |= kFlagRecompute;
+    if (above) v |= kFlagOutput;
+    if (above && !rec && !kept) v |= kFlagPadReuse;
+    *f = v;
+    above = above || rec;
+  }
+}
+
+// Ordered lists.  Rows [0, L*Bt): tokens of (layer, batch element) that enter the forward pass (recompute or
+// output); rows [L*Bt, L*Bt + Bt): the merged axis of a batch element (kept by any layer).  One CTA per row.
+__global__ void __launch_bounds__(kAlignThreads)
+align_lists_kernel(const uint8_t* __restrict__ flags, int32_t* __restrict__ run_ids, int32_t* __restrict__ run_len,
+                   int32_t* __restrict__ merged_ids, int32_t* __restrict__ merged_len, int L, int Bt, int L_tot,
+                   int run_capacity, int* __restrict__ d_status) {
+  __shared__ int warp_tot[kAlignThreads / 32];
+  const int row = blockIdx.x;
+  const bool is_run = row < L * Bt;
+  const int b = is_run ? row % Bt : row - L * Bt;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = (L_tot + kAlignThreads - 1) / kAlignThreads;
+  const int a = min(tid * per, L_tot), e = min(a + per, L_tot);
+  auto member = [&](int t) -> bool {
+    if (is_run) return (flags[(size_t)row * L_tot + t] & (kFlagRecompute | kFlagOutput)) != 0;
+    for (int n = 0; n < L; ++n)
+      if (flags[((size_t)n * Bt + b) * L_tot + t] & kFlagKept) return true;
+    return false;
+  };
+  int mine = 0;
+  for (int t = a; t < e; ++t) mine += member(t);
+  int inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  int before = 0, total = 0;
+  for (int i = 0; i < kAlignThreads / 32; ++i) {
+    if (i < warp) before += warp_tot[i];
+    total += warp_tot[i];
+  }
+  int pos = before + inc - mine;
+  int32_t* out = is_run ? run_ids + (size_t)row * run_capacity : merged_ids + (size_t)b * L_tot;
+  const int cap = is_run ? run_capacity : L_tot;
+  for (int t = a; t < e; ++t)
+    if (member(t)) {
+      if (pos < cap) out[pos] = t;
+      ++pos;
+    }
+  for (int i = total + tid; i < cap; i += kAlignThreads) out[i] = -1;          // unused tail of the list
+  if (tid == 0) {
+    if (is_run) run_len[row] = total; else merged_len[b] = total;
+    if (total > cap) atomicMax(d_status, (int)CHECK_LIST_CAPACITY);
+  }
+}
+
+cudaError_t launch_align(const samkv_shape_t& s, int L_tot, const int32_t* inv_map, const int32_t* tok_ids, int R,
+                         uint8_t* flags, int32_t* merged_ids, int32_t* merged_len, int32_t* run_ids, int run_capacity,
+                         int32_t* run_len, int* d_status, cudaStream_t stream) {
+  const int L = s.n_layers, Bt = s.batch;
+  cudaError_t e = cudaMemsetAsync(flags, 0, (size_t)L * Bt * L_tot, stream);
+  if (e != cudaSuccess) return e;
+  if (R > 0)
+    align_mark_kernel<<<(L * R + kAlignThreads - 1) / kAlignThreads, kAlignThreads, 0, stream>>>(tok_ids, flags, L, Bt, R,
+                                                                                              L_tot, d_status);
+  align_flags_kernel<<<dim3((L_tot + kAlignThreads - 1) / kAlignThreads, Bt), kAlignThreads, 0, stream>>>(
+      inv_map, flags, L, Bt, s.n_kv_heads, L_tot);
+  align_lists_kernel<<<L * Bt + Bt, kAlignThreads, 0, stream>>>(flags, run_ids, run_len, merged_ids, merged_len, L, Bt,
+                                                               L_tot, run_capacity, d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace samkv

@@ -447,4 +447,21 @@ samkv_status_t samkv_compact_units(samkv_handle_t handle, const samkv_shape_t* s
                                         static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_align(samkv_handle_t handle, const samkv_shape_t* shape, const int32_t* inv_map,
+                           const int32_t* tok_ids, int32_t R, uint8_t* flags_out, int32_t* merged_ids,
+                           int32_t* merged_len, int32_t* run_ids, int32_t run_capacity, int32_t* run_len, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (inv_map == nullptr || flags_out == nullptr || merged_ids == nullptr || merged_len == nullptr ||
+      run_ids == nullptr || run_len == nullptr)
+    return SAMKV_ERR_INVALID_ARG;
+  if (R < 0 || (R > 0 && tok_ids == nullptr) || run_capacity < 1) return SAMKV_ERR_INVALID_ARG;
+  return from_cuda(launch_align(*shape, lo.L_tot, inv_map, tok_ids, R, flags_out, merged_ids, merged_len, run_ids,
+                                run_capacity, run_len, h->d_status, static_cast<cudaStream_t>(stream)));
+}
+
 }  // extern "C"

@@ -60,6 +60,10 @@ cudaError_t launch_compact_units(const samkv_shape_t& s, const CtxTable& ct, con
                                  int S, void* Kc, void* Vc, int capacity, int32_t* cache_len, int32_t* inv_map,
                                  int* d_status, cudaStream_t stream);
 
+cudaError_t launch_align(const samkv_shape_t& s, int L_tot, const int32_t* inv_map, const int32_t* tok_ids, int R,
+                         uint8_t* flags, int32_t* merged_ids, int32_t* merged_len, int32_t* run_ids, int run_capacity,
+                         int32_t* run_len, int* d_status, cudaStream_t stream);
+
 struct AttnPlan {
   int n_splits;        // KV splits per (batch, kv head, row tile)
   int rows_per_cta;    // packed query rows (T_q * G) per CTA
@@ -76,7 +80,8 @@ enum DeviceCheck : int {
   CHECK_SEL_RANGE = 1,      // a selected unit id lies outside its context
   CHECK_APPEND_CAPACITY = 2, // cache_len + T_q exceeds the cache capacity
   CHECK_WAIT_TIMEOUT = 3,    // a bounded wait on an mbarrier ran out
-  CHECK_SMEM_ALIGNMENT = 4   // dynamic shared memory not aligned as the tensor-core tiles need
+  CHECK_SMEM_ALIGNMENT = 4,  // dynamic shared memory not aligned as the tensor-core tiles need
+  CHECK_LIST_CAPACITY = 5    // an output list is longer than the capacity the caller gave (it was truncated)
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
