@@ -148,6 +148,17 @@ samkv_status_t samkv_compact(samkv_handle_t h, const samkv_shape_t* shape, const
                              const int32_t* sel, const int32_t* k_units, void* Kc, void* Vc, int32_t cache_capacity,
                              int32_t* cache_len, int32_t* inv_map, void* stream);
 
+/* Composite cache of the protected positions only (Sec. 3.1 "Generate generic query vector": the initial and
+ * local K/V of all contexts, concatenated; also the "no-selection" ablation of Sec. 4.1).  Same result as
+ * samkv_select with k_units = protected units followed by samkv_compact, without scores or a unit list: the
+ * kept rows are two contiguous ranges per context.  The user query is then prefilled over it with samkv_attn
+ * (Kq/Vq appended), and the pooled Q of that pass is the Q_que that samkv_score takes.
+ * Arguments as for samkv_compact; cache_len is set to the protected token count (samkv_layout's kept tokens
+ * for k_units = protected units). */
+samkv_status_t samkv_compact_protected(samkv_handle_t h, const samkv_shape_t* shape, const void* K, const void* V,
+                                       void* Kc, void* Vc, int32_t cache_capacity, int32_t* cache_len,
+                                       int32_t* inv_map, void* stream);
+
 /* Write-back of recomputed rows (Sec. 3.3).  For every recomputed token r and every KV head that
  * kept it (slot = inv_map[l,b,h,tok_ids[l,r]] >= 0):
  *   overwrite: Kc[slot] = Knew[r], Vc[slot] = Vnew[r]

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "SAMKV_OK", 1: "SAMKV_ERR_INVALID_ARG", 2: "SAMKV_ERR_UNSUPPO
 EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll_status", "samkv_status_string",
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
            "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
-           "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align"]
+           "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected"]
 
 
 class SamkvError(RuntimeError):
@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
     L.samkv_select_cross_scratch_bytes.argtypes = [shp, i32p]
     L.samkv_select_cross_scratch_bytes.restype = ctypes.c_size_t
     L.samkv_align.argtypes = [vp, shp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp]
+    L.samkv_compact_protected.argtypes = [vp, shp, vp, vp, vp, vp, i32, vp, vp, vp]
     L.samkv_compact_units.argtypes = [vp, shp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("samkv_status_string", "samkv_workspace_bytes"):
@@ -277,3 +278,10 @@ def samkv_align(handle: Handle, shape: Shape, inv_map, tok_ids, flags_out, merge
     _check(lib().samkv_align(handle.h, shape.ref(), _ptr(inv_map), _ptr(tok_ids), R, _ptr(flags_out), _ptr(merged_ids),
                              _ptr(merged_len), _ptr(run_ids), int(run_ids.shape[-1]), _ptr(run_len), _stream()),
            "samkv_align")
+
+
+# ------------------------------------------------------------------ protected-only composite cache (Sec. 3.1)
+def samkv_compact_protected(handle: Handle, shape: Shape, K, V, Kc, Vc, cache_capacity: int, cache_len, inv_map=None):
+    _check(lib().samkv_compact_protected(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(Kc),
+                                         _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()),
+           "samkv_compact_protected")

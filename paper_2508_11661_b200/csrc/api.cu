@@ -294,6 +294,26 @@ samkv_status_t samkv_compact(samkv_handle_t handle, const samkv_shape_t* shape, 
                                   h->d_status, static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_compact_protected(samkv_handle_t handle, const samkv_shape_t* shape, const void* K, const void* V,
+                                       void* Kc, void* Vc, int32_t cache_capacity, int32_t* cache_len,
+                                       int32_t* inv_map, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (K == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || cache_len == nullptr) return SAMKV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc)) return SAMKV_ERR_INVALID_ARG;
+  SelTable sel;
+  int S = 0;
+  st = make_sel_table(shape, lo, lo.n_prot, &sel, &S);
+  if (st != SAMKV_OK) return st;
+  if (cache_capacity < S) return SAMKV_ERR_CAPACITY;
+  return from_cuda(launch_compact(*shape, lo.ct, sel, K, V, nullptr, Kc, Vc, cache_capacity, S, cache_len, inv_map,
+                                  h->d_status, static_cast<cudaStream_t>(stream)));
+}
+
 samkv_status_t samkv_update(samkv_handle_t handle, const samkv_shape_t* shape, void* Kc, void* Vc,
                             int32_t cache_capacity, const int32_t* inv_map, const int32_t* tok_ids, int32_t R,
                             const void* Knew, const void* Vnew, int32_t mode, void* stream) {

@@ -37,8 +37,9 @@ compact_kernel(const char* __restrict__ K, const char* __restrict__ V, const int
       const int c = find_segment(st.slot_off, ct.n_ctx, slot);
       const int r = slot - st.slot_off[c];
       const int j = r >> ct.block_shift;
-      const int unit = sel[slab * S_u + st.sel_off[c] + j];
-      const int m = unit - ct.unit_off[c];
+      // without a list (sel == nullptr) the kept units are the protected ones: two contiguous ranges per context
+      const int m = sel != nullptr ? sel[slab * S_u + st.sel_off[c] + j] - ct.unit_off[c]
+                                   : (j < st.n_init_units[c] ? j : st.first_local_unit[c] + (j - st.n_init_units[c]));
       const int t = ct.ctx_off[c] + (m << ct.block_shift) + (r & (ct.block_size - 1));
       if (m < 0 || m >= ct.unit_off[c + 1] - ct.unit_off[c] || t >= ct.ctx_off[c + 1]) {
         if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);
