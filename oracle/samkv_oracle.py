@@ -607,3 +607,28 @@ def align_layers(inv_map: np.ndarray, tok_ids: np.ndarray):
         run.append(np.asarray([t for t in range(L_tot) if flags[n, t] & (FLAG_RECOMPUTE | FLAG_OUTPUT)],
                               dtype=np.int64))
     return flags, np.asarray(merged, dtype=np.int64), run
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.2: "each block is represented by the mean vector of its constituent token caches"
+# --------------------------------------------------------------------------------------
+def block_means(K: np.ndarray, ctx_offsets, B: int, dtype: str | None = None) -> np.ndarray:
+    """Kbar[h, u, :] = mean of K[h, t, :] over the tokens t of unit u (a short tail unit averages
+    the tokens it has).  K: [Hkv, L_tot, d] float64 -> [Hkv, U_tot, d]; `dtype` ("bf16" / "f32")
+    rounds the result once to the storage type of the representative cache, None keeps float64.
+    Scoring a query against Kbar with `token_scores` over the unit offsets gives the block scores."""
+    K = np.asarray(K, dtype=F64)
+    nb, unit_off = unit_layout(ctx_offsets, B)
+    Hkv, _, d = K.shape
+    out = np.zeros((Hkv, unit_off[-1], d), dtype=F64)
+    for h in range(Hkv):
+        for c in range(len(nb)):
+            lo, hi = int(ctx_offsets[c]), int(ctx_offsets[c + 1])
+            for m in range(nb[c]):
+                a = lo + m * B
+                b = min(a + B, hi)
+                acc = np.zeros(d, dtype=F64)
+                for t in range(a, b):
+                    acc += K[h, t]
+                out[h, unit_off[c] + m] = acc / (b - a)
+    return out if dtype is None else round_to_dtype(out, dtype)

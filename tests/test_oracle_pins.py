@@ -641,3 +641,43 @@ def test_align_layers_without_recomputation_only_marks_kept_tokens():
     flags, merged, run = O.align_layers(inv, np.full((3, 4), -1))
     assert flags.sum() == 2 and flags[0, 2] == O.FLAG_KEPT and flags[2, 7] == O.FLAG_KEPT
     assert merged.tolist() == [2, 7] and all(len(x) == 0 for x in run)
+
+
+# ------------------------------------------------------------------------------------------
+# Section 3.2: blocks represented by the mean vector of their token caches
+# ------------------------------------------------------------------------------------------
+def test_block_means_hand_values_tail_and_token_mode():
+    K = np.zeros((1, 5, 2))
+    K[0] = [[1, 2], [3, 6], [10, 20], [30, 40], [7, 9]]
+    off = [0, 2, 5]                                              # contexts of 2 and 3 tokens
+    Kb = O.block_means(K, off, 2)
+    assert Kb.shape == (1, 3, 2)
+    assert Kb[0].tolist() == [[2, 4], [20, 30], [7, 9]]          # the short tail unit is its single token
+    assert np.array_equal(O.block_means(K, off, 1), K)           # token mode: the representative is the key itself
+    Kb4 = O.block_means(K, off, 4)                               # units never cross a context boundary
+    assert Kb4[0].tolist() == [[2, 4], [47 / 3, 23]]
+
+
+@pytest.mark.parametrize("B", [2, 8, 64])
+def test_score_on_block_means_equals_block_mean_of_token_scores(B):
+    """<q, mean_t K_t> = mean_t <q, K_t>: scoring the representatives reproduces the unit scores."""
+    r = np.random.default_rng(B)
+    lens = [130, 64, 7, 200]
+    off = [0] + list(np.cumsum(lens))
+    Hkv, d = 2, 16
+    K = r.normal(size=(Hkv, off[-1], d))
+    q = r.normal(size=(len(lens), Hkv, d))
+    u_tok = O.unit_scores(O.token_scores(q, K, off), off, B)
+    nb, unit_off = O.unit_layout(off, B)
+    u_rep = O.token_scores(q, O.block_means(K, off, B), unit_off)
+    assert np.allclose(u_tok, u_rep, rtol=0, atol=1e-12)
+
+
+def test_block_means_rounding_to_storage_type():
+    r = np.random.default_rng(5)
+    K = O.round_to_bf16(r.normal(size=(1, 64, 8)))
+    exact = O.block_means(K, [0, 64], 16)
+    stored = O.block_means(K, [0, 64], 16, "bf16")
+    assert np.array_equal(stored, O.round_to_bf16(stored))                     # representable
+    assert (np.abs(stored - exact) <= 2.0 ** -8 * np.abs(exact)).all()   # half a bf16 ulp: 8 significant bits
+    assert np.array_equal(O.block_means(K, [0, 64], 16, "f32"), exact.astype(np.float32).astype(np.float64))
