@@ -239,6 +239,21 @@ samkv_status_t samkv_compact_units(samkv_handle_t h, const samkv_shape_t* shape,
                                    const int32_t* sel, int32_t S_u, void* Kc, void* Vc, int32_t cache_capacity,
                                    int32_t* cache_len, int32_t* inv_map, void* stream);
 
+/* ---- block representatives (Sec. 3.2: "each block is represented by the mean vector of its token caches") --- */
+
+/* Kbar[l,b,h,u,:] = mean over the tokens of unit u of K[l,b,h,t,:] (fp32 sum in a fixed order, one rounding to the
+ * storage dtype; a short tail unit averages the tokens it has).  Query-independent: run once per stored document.
+ *   K    [L, Bt, Hkv, L_tot, d]      Kbar [L, Bt, Hkv, U_tot, d], same dtype, 16-byte aligned */
+samkv_status_t samkv_block_means(samkv_handle_t h, const samkv_shape_t* shape, const void* K, void* Kbar, void* stream);
+
+/* samkv_score on the representatives: scores[l,b,h,u] = <q^_c, Kbar[l,b,h,u,:]> for u in context c, which equals
+ * the block-mean of the token scores up to the one rounding of Kbar (inner products are linear).  Reads d*e bytes
+ * per unit instead of per token.  Other arguments, outputs and errors as for samkv_score; `shape` is the token-level
+ * shape (block_size = B), the same one samkv_select / samkv_compact take afterwards. */
+samkv_status_t samkv_score_blocks(samkv_handle_t h, const samkv_shape_t* shape, const void* Kbar, const void* Q,
+                                  int32_t T_q, const void* Qloc, int32_t T_loc, int32_t use_bias, float* scores_out,
+                                  float* qhat_out, void* stream);
+
 /* ---- cross-layer alignment of the sparse caches (Sec. 3.3 "Recomputation") ------------------------ */
 
 #define SAMKV_FLAG_KEPT 1       /* some KV head of the layer keeps the token (not a blank position) */

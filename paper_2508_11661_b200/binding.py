@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "SAMKV_OK", 1: "SAMKV_ERR_INVALID_ARG", 2: "SAMKV_ERR_UNSUPPO
 EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll_status", "samkv_status_string",
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
            "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
-           "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected"]
+           "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected",
+           "samkv_block_means", "samkv_score_blocks"]
 
 
 class SamkvError(RuntimeError):
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
     L.samkv_select_cross_scratch_bytes.restype = ctypes.c_size_t
     L.samkv_align.argtypes = [vp, shp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp]
     L.samkv_compact_protected.argtypes = [vp, shp, vp, vp, vp, vp, i32, vp, vp, vp]
+    L.samkv_block_means.argtypes = [vp, shp, vp, vp, vp]
+    L.samkv_score_blocks.argtypes = L.samkv_score.argtypes
     L.samkv_compact_units.argtypes = [vp, shp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("samkv_status_string", "samkv_workspace_bytes"):
@@ -285,3 +288,14 @@ def samkv_compact_protected(handle: Handle, shape: Shape, K, V, Kc, Vc, cache_ca
     _check(lib().samkv_compact_protected(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(Kc),
                                          _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()),
            "samkv_compact_protected")
+
+
+# ------------------------------------------------------------------ block representatives (Sec. 3.2)
+def samkv_block_means(handle: Handle, shape: Shape, K, Kbar):
+    _check(lib().samkv_block_means(handle.h, shape.ref(), _ptr(K), _ptr(Kbar), _stream()), "samkv_block_means")
+
+
+def samkv_score_blocks(handle: Handle, shape: Shape, Kbar, Q, T_q: int, Qloc, T_loc: int, use_bias: int, scores_out,
+                       qhat_out=None):
+    _check(lib().samkv_score_blocks(handle.h, shape.ref(), _ptr(Kbar), _ptr(Q), T_q, _ptr(Qloc), T_loc, use_bias,
+                                    _ptr(scores_out), _ptr(qhat_out), _stream()), "samkv_score_blocks")

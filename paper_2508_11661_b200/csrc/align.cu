@@ -25,27 +25,47 @@ align_mark_kernel(const int32_t* __restrict__ tok_ids, uint8_t* __restrict__ fla
   for (int b = 0; b < Bt; ++b) flags[((size_t)n * Bt + b) * L_tot + t] = kFlagRecompute;
 }
 
-// One thread per (batch element, token), layers from the top down: rule 1 propagates "recomputed above".
+// One thread per (layer, batch element, token): is the token kept by any head, and is its listing effective.
 __global__ void __launch_bounds__(kAlignThreads)
-align_flags_kernel(const int32_t* __restrict__ inv_map, uint8_t* __restrict__ flags, int L, int Bt, int Hkv, int L_tot) {
+align_kept_kernel(const int32_t* __restrict__ inv_map, uint8_t* __restrict__ flags, int Hkv, int L_tot) {
+  const int t = blockIdx.x * kAlignThreads + threadIdx.x;
+  const size_t lb = blockIdx.y;                                 // layer * Bt + batch element
+  if (t >= L_tot) return;
+  const int32_t* row = inv_map + lb * Hkv * L_tot + t;
+  bool kept = false;
+  for (int h = 0; h < Hkv; ++h) kept = kept || (row[(size_t)h * L_tot] >= 0);
+  uint8_t* f = flags + lb * L_tot + t;
+  const bool rec = (*f != 0) && kept;
+  *f = (kept ? kFlagKept : 0) | (rec ? kFlagRecompute : 0);
+}
+
+// One thread per (batch element, token), layers from the top down: rule 1 propagates "recomputed above".
+// Layer 0's byte also carries, in kScratchOnAxis, "kept by some layer" for the list kernel; it is cleared afterwards.
+constexpr uint8_t kScratchOnAxis = 0x80;
+__global__ void __launch_bounds__(kAlignThreads)
+align_rules_kernel(uint8_t* __restrict__ flags, int L, int Bt, int L_tot) {
   const int t = blockIdx.x * kAlignThreads + threadIdx.x;
   const int b = blockIdx.y;
   if (t >= L_tot) return;
-  bool above = false;                                           // some higher layer recomputes the token
+  bool above = false, on_axis = false;                          // some higher layer recomputes / any layer keeps
+#pragma unroll 4
   for (int n = L - 1; n >= 0; --n) {
-    bool kept = false;
-    const int32_t* row = inv_map + (((size_t)n * Bt + b) * Hkv) * L_tot + t;
-    for (int h = 0; h < Hkv; ++h) kept = kept || (row[(size_t)h * L_tot] >= 0);
     uint8_t* f = flags + ((size_t)n * Bt + b) * L_tot + t;
-    const bool rec = (*f != 0) && kept;
-    uint8_t v = 0;
-    if (kept) v |= kFlagKept;
-    if (rec) v |= kFlagRecompute;
+    uint8_t v = *f;
+    const bool kept = v & kFlagKept, rec = v & kFlagRecompute;
     if (above) v |= kFlagOutput;
     if (above && !rec && !kept) v |= kFlagPadReuse;
-    *f = v;
     above = above || rec;
+    on_axis = on_axis || kept;
+    if (n == 0 && on_axis) v |= kScratchOnAxis;
+    *f = v;
   }
+}
+
+__global__ void __launch_bounds__(kAlignThreads)
+align_clear_kernel(uint8_t* __restrict__ flags, int n) {        // layer 0 occupies the first Bt * L_tot bytes
+  const int i = blockIdx.x * kAlignThreads + threadIdx.x;
+  if (i < n) flags[i] &= (uint8_t)~kScratchOnAxis;
 }
 
 // Ordered lists.  Rows [0, L*Bt): tokens of (layer, batch element) that enter the forward pass (recompute or
@@ -63,9 +83,7 @@ align_lists_kernel(const uint8_t* __restrict__ flags, int32_t* __restrict__ run_
   const int a = min(tid * per, L_tot), e = min(a + per, L_tot);
   auto member = [&](int t) -> bool {
     if (is_run) return (flags[(size_t)row * L_tot + t] & (kFlagRecompute | kFlagOutput)) != 0;
-    for (int n = 0; n < L; ++n)
-      if (flags[((size_t)n * Bt + b) * L_tot + t] & kFlagKept) return true;
-    return false;
+    return (flags[(size_t)b * L_tot + t] & kScratchOnAxis) != 0;
   };
   int mine = 0;
   for (int t = a; t < e; ++t) mine += member(t);
@@ -101,15 +119,18 @@ cudaError_t launch_align(const samkv_shape_t& s, int L_tot, const int32_t* inv_m
                          uint8_t* flags, int32_t* merged_ids, int32_t* merged_len, int32_t* run_ids, int run_capacity,
                          int32_t* run_len, int* d_status, cudaStream_t stream) {
   const int L = s.n_layers, Bt = s.batch;
+  if ((long long)L * Bt > 65535) return cudaErrorInvalidConfiguration;      // (layer, batch) pairs ride on gridDim.y
   cudaError_t e = cudaMemsetAsync(flags, 0, (size_t)L * Bt * L_tot, stream);
   if (e != cudaSuccess) return e;
   if (R > 0)
     align_mark_kernel<<<(L * R + kAlignThreads - 1) / kAlignThreads, kAlignThreads, 0, stream>>>(tok_ids, flags, L, Bt, R,
                                                                                               L_tot, d_status);
-  align_flags_kernel<<<dim3((L_tot + kAlignThreads - 1) / kAlignThreads, Bt), kAlignThreads, 0, stream>>>(
-      inv_map, flags, L, Bt, s.n_kv_heads, L_tot);
+  const unsigned tiles = (L_tot + kAlignThreads - 1) / kAlignThreads;
+  align_kept_kernel<<<dim3(tiles, L * Bt), kAlignThreads, 0, stream>>>(inv_map, flags, s.n_kv_heads, L_tot);
+  align_rules_kernel<<<dim3(tiles, Bt), kAlignThreads, 0, stream>>>(flags, L, Bt, L_tot);
   align_lists_kernel<<<L * Bt + Bt, kAlignThreads, 0, stream>>>(flags, run_ids, run_len, merged_ids, merged_len, L, Bt,
                                                                L_tot, run_capacity, d_status);
+  align_clear_kernel<<<(Bt * L_tot + kAlignThreads - 1) / kAlignThreads, kAlignThreads, 0, stream>>>(flags, Bt * L_tot);
   return cudaGetLastError();
 }
 

@@ -467,6 +467,33 @@ samkv_status_t samkv_compact_units(samkv_handle_t handle, const samkv_shape_t* s
                                         static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_block_means(samkv_handle_t handle, const samkv_shape_t* shape, const void* K, void* Kbar,
+                                 void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (K == nullptr || Kbar == nullptr || !aligned16(K) || !aligned16(Kbar)) return SAMKV_ERR_INVALID_ARG;
+  return from_cuda(launch_block_means(*shape, lo.ct, K, Kbar, h->sm_count, static_cast<cudaStream_t>(stream)));
+}
+
+samkv_status_t samkv_score_blocks(samkv_handle_t handle, const samkv_shape_t* shape, const void* Kbar, const void* Q,
+                                  int32_t T_q, const void* Qloc, int32_t T_loc, int32_t use_bias, float* scores_out,
+                                  float* qhat_out, void* stream) {
+  Layout lo;
+  samkv_status_t st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  // the representatives form a cache of their own with one "token" per unit
+  samkv_shape_t units = *shape;
+  units.ctx_offsets = lo.ct.unit_off;
+  units.block_size = 1;
+  units.n_init = shape->n_init / shape->block_size;
+  units.n_local = shape->n_local / shape->block_size;
+  return samkv_score(handle, &units, Kbar, Q, T_q, Qloc, T_loc, use_bias, scores_out, qhat_out, stream);
+}
+
 samkv_status_t samkv_align(samkv_handle_t handle, const samkv_shape_t* shape, const int32_t* inv_map,
                            const int32_t* tok_ids, int32_t R, uint8_t* flags_out, int32_t* merged_ids,
                            int32_t* merged_len, int32_t* run_ids, int32_t run_capacity, int32_t* run_len, void* stream) {

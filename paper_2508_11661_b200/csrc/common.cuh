@@ -64,6 +64,9 @@ cudaError_t launch_align(const samkv_shape_t& s, int L_tot, const int32_t* inv_m
                          uint8_t* flags, int32_t* merged_ids, int32_t* merged_len, int32_t* run_ids, int run_capacity,
                          int32_t* run_len, int* d_status, cudaStream_t stream);
 
+cudaError_t launch_block_means(const samkv_shape_t& s, const CtxTable& ct, const void* K, void* Kbar, int sm_count,
+                               cudaStream_t stream);
+
 struct AttnPlan {
   int n_splits;        // KV splits per (batch, kv head, row tile)
   int rows_per_cta;    // packed query rows (T_q * G) per CTA
