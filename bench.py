@@ -290,9 +290,11 @@ class Pipeline:
         self.decode_graph.replay()
 
     def launches_per_step(self) -> int:
-        n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + KERNELS_PER_CALL["compact"]
+        per_group = KERNELS_PER_CALL["compact"]
         if self.R > 0:
-            n += KERNELS_PER_CALL["update"]
+            per_group += KERNELS_PER_CALL["update"]
+        # the timed schedule gathers and updates group by group
+        n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + self.groups * per_group
         n += self.w.n_layers * KERNELS_PER_CALL["attn_append_split"]
         return n + self.w.n_layers * self.w.decode_steps * KERNELS_PER_CALL["attn_append_split"]
 

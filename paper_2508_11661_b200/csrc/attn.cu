@@ -76,6 +76,7 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
 __global__ void append_kernel(char* __restrict__ Kc, char* __restrict__ Vc, const int32_t* __restrict__ cache_len,
                               const char* __restrict__ Kq, const char* __restrict__ Vq, int Hkv, int T_q, int capacity,
                               int row_bytes, long long n_threads, int* __restrict__ d_status) {
+  pdl_launch_dependents();      // the attention kernel may set itself up while the chunk is being appended
   const int lanes = row_bytes / 16;
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= n_threads) return;
@@ -210,6 +211,7 @@ attn_finalize_kernel(const float* __restrict__ part_o, const float2* __restrict_
   constexpr int kEpl = kHeadDim / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * 4 + warp;
+  pdl_wait();                   // the attention kernel's partials and its reads of cache_len are complete
   if (n_splits > 1 && row < n_rows) {
     float M = kNegInf;
     for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[row * n_splits + s].x);
@@ -286,8 +288,21 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   }
   if (plan.n_splits > 1 || appended) {
     const long long blocks = plan.n_splits > 1 ? (long long)((out_rows + 3) / 4) : 1;
-    attn_finalize_kernel<T, kHeadDim><<<(unsigned)blocks, 128, 0, stream>>>(
-        part_o, part_ml, (T*)O, lse, len_l, Bt, Hq, T_q, capacity, appended, plan.n_splits, (long long)out_rows);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    if (sizeof(T) == 2 && plan.rows_per_cta == 256) {     // the tensor-memory kernel releases its dependents early
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+    }
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_finalize_kernel<T, kHeadDim>, (const float*)part_o,
+                                       (const float2*)part_ml, (T*)O, lse, len_l, Bt, Hq, T_q, capacity, appended,
+                                       plan.n_splits, (long long)out_rows);
+    if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }

@@ -275,6 +275,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
   if (warp == kLoadWarp) {
     // ================= loader: K ring and V ring =================
+    pdl_wait();                 // rows appended by the kernel before this one are in the cache from here on
     for (int j = 0; j < nt; ++j) {
       const int s = j % kStages;
       const uint32_t round = (uint32_t)(j / kStages);
@@ -494,6 +495,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   // ---- teardown: every role arrives here, then the allocating warp frees tensor memory ----
   tc_fence_before();
   __syncthreads();
+  pdl_launch_dependents();      // results are written: the merge kernel may be scheduled (it still waits for our exit)
   if (tid == 0 && *s_fail) atomicMax(d_status, (int)CHECK_WAIT_TIMEOUT);
   if (warp == kMmaWarp) {
     tc_fence_after();
@@ -548,10 +550,21 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::kSmemBytes);
   if (e != cudaSuccess) return e;
-  attn_tc2_kernel<<<(unsigned)blocks, tc2::kThreads, tc2::kSmemBytes, stream>>>(
-      tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (__nv_bfloat16*)O, lse, part_o, part_ml, s.n_q_heads, s.n_kv_heads,
-      T_q, capacity, appended, scale, plan.n_splits, row_tiles, d_status);
-  return cudaGetLastError();
+  // Launched so that it may start while the kernel before it in the stream (the append of the chunk) is still
+  // running: set-up and the Q loads need nothing from it; the loader waits before its first K/V tile.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks);
+  cfg.blockDim = dim3(tc2::kThreads);
+  cfg.dynamicSmemBytes = tc2::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attn_tc2_kernel, tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (__nv_bfloat16*)O, lse,
+                            part_o, part_ml, s.n_q_heads, s.n_kv_heads, T_q, capacity, appended, scale, plan.n_splits,
+                            row_tiles, d_status);
 }
 
 }  // namespace samkv

@@ -130,6 +130,12 @@ __device__ __forceinline__ void st_stream(void* p, const uint4& v) {
   asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization attribute may start
+// once every CTA of the kernel before it in the stream has called pdl_launch_dependents() (or exited); it must call
+// pdl_wait() before touching anything that kernel writes.  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Context that owns global index `x` in a prefix table `off[0..n]` (off[c] <= x < off[c+1]).
 __device__ __forceinline__ int find_segment(const int* off, int n, int x) {
   int lo = 0, hi = n - 1;

@@ -20,39 +20,115 @@ __device__ __forceinline__ float warp_sum(float v) {
 // ------------------------------------------------------------------------------------------------
 // Q_que = mean_t Q (Sec. 3.1), q_loc_j = mean_t Qloc_j, Eq. 1, then the mean over the G query heads
 // of a KV group.  One CTA per (layer, batch, kv head) with one warp per query head of the group; a lane
-// owns kEpl = d/32 consecutive elements, so the cosines need warp shuffles only (no block barriers
-// on the dependent chain).  The sum over j != i is formed as (sum over all j) - (own term); fp32.
+// owns kEpl = d/32 consecutive elements (one vector load per row), so the cosines need warp shuffles
+// only.  The kernel is latency-bound (a few KB per CTA), so independent work is batched: the local
+// queries of kQhatBatch contexts are loaded and reduced together, and the GQA fold runs on chunks of
+// contexts between two block barriers.  The sum over j != i is formed as (sum over all j) - (own
+// term); fp32 throughout, fixed summation order.
 //   qhat [L*Bt, D, Hkv, d]
 // ------------------------------------------------------------------------------------------------
+constexpr int kQhatBatch = 4;               // contexts whose local queries are in flight together
+constexpr int kQhatFoldBytes = 16 * 1024;   // shared memory for one chunk of per-head Q^_i vectors
+
 template <typename T, int kEpl>
-__global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc, float* __restrict__ qhat, int T_q,
-                            int T_loc, int Hq, int Hkv, int D, int use_bias) {
+__device__ __forceinline__ void load_row_slice(const T* p, float* out) {      // kEpl consecutive elements, one load
+  if constexpr (sizeof(T) == 4) {
+    if constexpr (kEpl == 4) {
+      const float4 v = *reinterpret_cast<const float4*>(p);
+      out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+    } else {
+      const float2 v = *reinterpret_cast<const float2*>(p);
+      out[0] = v.x; out[1] = v.y;
+    }
+  } else {
+    if constexpr (kEpl == 4) {
+      const uint2 v = *reinterpret_cast<const uint2*>(p);
+      out[0] = bf16_lo(v.x); out[1] = bf16_hi(v.x); out[2] = bf16_lo(v.y); out[3] = bf16_hi(v.y);
+    } else {
+      const uint32_t v = *reinterpret_cast<const uint32_t*>(p);
+      out[0] = bf16_lo(v); out[1] = bf16_hi(v);
+    }
+  }
+}
+
+// kMaxThreads bounds G * 32; the register cap that comes with it keeps at least 7 / 3 / 1 CTAs of 128 / 256 / 1024
+// threads on an SM, so that a grid of about a thousand CTAs is resident in one wave.
+template <typename T, int kEpl, int kMaxThreads>
+__global__ void __launch_bounds__(kMaxThreads, kMaxThreads == 128 ? 7 : (kMaxThreads == 256 ? 3 : 1))
+qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc, float* __restrict__ qhat, int T_q,
+                            int T_loc, int Hq, int Hkv, int D, int use_bias, int fold_ctx) {
   constexpr int d = kEpl * 32;
   extern __shared__ float smem[];
   const int G = Hq / Hkv;
   float* w_all = smem;                       // [G][D] |cos| weights
-  float* fold = smem + G * D;                // [G][d] per-head Q^_i of the context being folded
+  float* fold = smem + G * D;                // [fold_ctx][G][d] per-head Q^_i of a chunk of contexts
   const int h = blockIdx.x % Hkv;
   const size_t lb = blockIdx.x / Hkv;
   const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int hq = h * G + g;
   const bool bias = use_bias && Qloc != nullptr && D > 1;
   float* w = w_all + g * D;
+  const size_t row_stride = (size_t)Hq * d;
 
-  auto pooled = [&](const T* base, int T_n, size_t stride, float* out) {   // mean over T_n rows, summed in row order
+  // mean over T_n rows, summed in row order; the loads of kRowsInFlight rows are issued before their sums
+  constexpr int kRowsInFlight = 8;
+  auto pooled = [&](const T* base, int T_n, float* out) {
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) out[i] = 0.f;
-#pragma unroll 8
-    for (int t = 0; t < T_n; ++t) {
+    for (int t0 = 0; t0 < T_n; t0 += kRowsInFlight) {
+      float r[kRowsInFlight][kEpl];
 #pragma unroll
-      for (int i = 0; i < kEpl; ++i) out[i] += load_as_float(base + t * stride + lane * kEpl + i);
+      for (int u = 0; u < kRowsInFlight; ++u)
+        if (t0 + u < T_n) load_row_slice<T, kEpl>(base + (t0 + u) * row_stride + lane * kEpl, r[u]);
+#pragma unroll
+      for (int u = 0; u < kRowsInFlight; ++u)
+        if (t0 + u < T_n) {
+#pragma unroll
+          for (int i = 0; i < kEpl; ++i) out[i] += r[u][i];
+        }
     }
+    if (T_n > 1) {
 #pragma unroll
-    for (int i = 0; i < kEpl; ++i) out[i] = out[i] / (float)T_n;
+      for (int i = 0; i < kEpl; ++i) out[i] = out[i] / (float)T_n;
+    }
+  };
+  auto qloc_row = [&](int j) { return Qloc + ((lb * D + j) * T_loc * Hq + hq) * d; };
+  // local queries of contexts j0 .. j0 + kQhatBatch - 1 (zero past the last context): the rows of the batch are
+  // loaded together, so that a batch costs one memory round trip per local row rather than one per context
+  auto pooled_batch = [&](int j0, int j_end, float (*ql)[kEpl]) {
+#pragma unroll
+    for (int u = 0; u < kQhatBatch; ++u) {
+#pragma unroll
+      for (int i = 0; i < kEpl; ++i) ql[u][i] = 0.f;
+    }
+    for (int t = 0; t < T_loc; ++t) {
+      float r[kQhatBatch][kEpl];
+#pragma unroll
+      for (int u = 0; u < kQhatBatch; ++u) {
+        if (j0 + u < j_end) {
+          load_row_slice<T, kEpl>(qloc_row(j0 + u) + t * row_stride + lane * kEpl, r[u]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < kEpl; ++i) r[u][i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kQhatBatch; ++u) {
+#pragma unroll
+        for (int i = 0; i < kEpl; ++i) ql[u][i] += r[u][i];
+      }
+    }
+    if (T_loc > 1) {
+#pragma unroll
+      for (int u = 0; u < kQhatBatch; ++u) {
+#pragma unroll
+        for (int i = 0; i < kEpl; ++i) ql[u][i] = ql[u][i] / (float)T_loc;
+      }
+    }
   };
 
   float qq[kEpl], S[kEpl];
-  pooled(Q + (lb * T_q * Hq + hq) * d, T_q, (size_t)Hq * d, qq);
+  pooled(Q + (lb * T_q * Hq + hq) * d, T_q, qq);
 #pragma unroll
   for (int i = 0; i < kEpl; ++i) S[i] = 0.f;
   if (bias) {
@@ -60,51 +136,63 @@ __global__ void qhat_kernel(const T* __restrict__ Q, const T* __restrict__ Qloc,
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) na2 = fmaf(qq[i], qq[i], na2);
     na2 = warp_sum(na2);
-#pragma unroll 4
-    for (int j = 0; j < D; ++j) {
-      float ql[kEpl];
-      pooled(Qloc + ((lb * D + j) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql);
-      float dot = 0.f, nb2 = 0.f;
+    for (int j0 = 0; j0 < D; j0 += kQhatBatch) {
+      float ql[kQhatBatch][kEpl], dot[kQhatBatch], nb2[kQhatBatch];
+      pooled_batch(j0, D, ql);
 #pragma unroll
-      for (int i = 0; i < kEpl; ++i) { dot = fmaf(qq[i], ql[i], dot); nb2 = fmaf(ql[i], ql[i], nb2); }
-      dot = warp_sum(dot);
-      nb2 = warp_sum(nb2);
-      const float wj = (na2 > 0.f && nb2 > 0.f) ? fabsf(dot) / (sqrtf(na2) * sqrtf(nb2)) : 0.f;
-      if (lane == 0) w[j] = wj;
+      for (int u = 0; u < kQhatBatch; ++u) {
+        dot[u] = nb2[u] = 0.f;
 #pragma unroll
-      for (int i = 0; i < kEpl; ++i) S[i] = fmaf(wj, ql[i], S[i]);
+        for (int i = 0; i < kEpl; ++i) { dot[u] = fmaf(qq[i], ql[u][i], dot[u]); nb2[u] = fmaf(ql[u][i], ql[u][i], nb2[u]); }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {                       // 2 * kQhatBatch independent shuffle chains
+#pragma unroll
+        for (int u = 0; u < kQhatBatch; ++u) {
+          dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], o);
+          nb2[u] += __shfl_xor_sync(0xffffffffu, nb2[u], o);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kQhatBatch; ++u) {                    // S accumulates in context order
+        if (j0 + u < D) {
+          const float wj = (na2 > 0.f && nb2[u] > 0.f) ? fabsf(dot[u]) / (sqrtf(na2) * sqrtf(nb2[u])) : 0.f;
+          if (lane == 0) w[j0 + u] = wj;
+#pragma unroll
+          for (int i = 0; i < kEpl; ++i) S[i] = fmaf(wj, ql[u][i], S[i]);
+        }
+      }
     }
     __syncwarp();
   }
   const float inv_dm1 = bias ? 1.0f / (float)(D - 1) : 0.f;
   float* out = qhat + (lb * D * Hkv + h) * d;            // + i * Hkv * d
-  float ql_cur[kEpl], ql_nxt[kEpl];
+  for (int c0 = 0; c0 < D; c0 += fold_ctx) {
+    const int nc = min(fold_ctx, D - c0);
+    for (int ci0 = 0; ci0 < nc; ci0 += kQhatBatch) {
+      float ql[kQhatBatch][kEpl];
+      if (bias) pooled_batch(c0 + ci0, c0 + nc, ql);       // second read of the rows: served by the caches
 #pragma unroll
-  for (int i = 0; i < kEpl; ++i) ql_cur[i] = ql_nxt[i] = 0.f;
-  if (bias) pooled(Qloc + ((lb * D + 0) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql_cur);
-  for (int i0 = 0; i0 < D; ++i0) {
-    // fetch the next context's local query before the barriers of this one
-    if (bias && i0 + 1 < D) pooled(Qloc + ((lb * D + i0 + 1) * T_loc * Hq + hq) * d, T_loc, (size_t)Hq * d, ql_nxt);
-    float val[kEpl];
+      for (int u = 0; u < kQhatBatch; ++u) {
+        if (ci0 + u < nc) {
+          const float wi = bias ? w[c0 + ci0 + u] : 0.f;
 #pragma unroll
-    for (int i = 0; i < kEpl; ++i) val[i] = qq[i];
-    if (bias) {
-      const float wi = w[i0];
-#pragma unroll
-      for (int i = 0; i < kEpl; ++i) val[i] += (S[i] - wi * ql_cur[i]) * inv_dm1;
+          for (int i = 0; i < kEpl; ++i) {
+            const float val = bias ? qq[i] + (S[i] - wi * ql[u][i]) * inv_dm1 : qq[i];
+            fold[((ci0 + u) * G + g) * d + lane * kEpl + i] = val;
+          }
+        }
+      }
     }
-#pragma unroll
-    for (int i = 0; i < kEpl; ++i) fold[g * d + lane * kEpl + i] = val[i];
     __syncthreads();
     // mean over the G query heads of the group, summed in head order
-    for (int e = threadIdx.x; e < d; e += blockDim.x) {
-      float acc = fold[e];
-      for (int gg = 1; gg < G; ++gg) acc += fold[gg * d + e];
-      out[(size_t)i0 * Hkv * d + e] = acc / (float)G;
+    for (int e = threadIdx.x; e < nc * d; e += blockDim.x) {
+      const int ci = e / d, x = e - ci * d;
+      float acc = fold[(ci * G) * d + x];
+      for (int gg = 1; gg < G; ++gg) acc += fold[(ci * G + gg) * d + x];
+      out[(size_t)(c0 + ci) * Hkv * d + x] = acc / (float)G;
     }
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < kEpl; ++i) ql_cur[i] = ql_nxt[i];
   }
 }
 
@@ -113,15 +201,24 @@ cudaError_t launch_qhat(const samkv_shape_t& s, const void* Q, int T_q, const vo
   const int blocks = s.n_layers * s.batch * s.n_kv_heads;
   const int G = s.n_q_heads / s.n_kv_heads;
   if (G > 32) return cudaErrorInvalidConfiguration;        // one warp per query head of a group
-  const size_t smem = (size_t)(G * s.n_ctx + G * s.head_dim) * sizeof(float);
+  int fold_ctx = kQhatFoldBytes / (G * s.head_dim * (int)sizeof(float));
+  fold_ctx = fold_ctx < 1 ? 1 : (fold_ctx > s.n_ctx ? s.n_ctx : fold_ctx);
+  const size_t smem = (size_t)(G * s.n_ctx + fold_ctx * G * s.head_dim) * sizeof(float);
+#define SAMKV_QHAT_N(T, EPL, N)                                                                                  \
+  qhat_kernel<T, EPL, N><<<blocks, G * 32, smem, stream>>>((const T*)Q, (const T*)Qloc, qhat, T_q, T_loc,          \
+                                                           s.n_q_heads, s.n_kv_heads, s.n_ctx, use_bias, fold_ctx)
 #define SAMKV_QHAT(T, EPL)                                                                                        \
-  qhat_kernel<T, EPL><<<blocks, G * 32, smem, stream>>>((const T*)Q, (const T*)Qloc, qhat, T_q, T_loc, s.n_q_heads, \
-                                                        s.n_kv_heads, s.n_ctx, use_bias)
+  do {                                                                                                            \
+    if (G <= 4) SAMKV_QHAT_N(T, EPL, 128);                                                                        \
+    else if (G <= 8) SAMKV_QHAT_N(T, EPL, 256);                                                                   \
+    else SAMKV_QHAT_N(T, EPL, 1024);                                                                              \
+  } while (0)
   if (s.dtype == SAMKV_BF16) {
     if (s.head_dim == 128) SAMKV_QHAT(__nv_bfloat16, 4); else SAMKV_QHAT(__nv_bfloat16, 2);
   } else {
     if (s.head_dim == 128) SAMKV_QHAT(float, 4); else SAMKV_QHAT(float, 2);
   }
+#undef SAMKV_QHAT_N
 #undef SAMKV_QHAT
   return cudaGetLastError();
 }
