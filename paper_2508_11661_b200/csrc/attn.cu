@@ -213,23 +213,62 @@ attn_finalize_kernel(const float* __restrict__ part_o, const float2* __restrict_
   const long long row = (long long)blockIdx.x * 4 + warp;
   pdl_wait();                   // the attention kernel's partials and its reads of cache_len are complete
   if (n_splits > 1 && row < n_rows) {
-    float M = kNegInf;
-    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[row * n_splits + s].x);
+    // lane s holds (m, l) of split s (and of split s + 32): one round trip for all of them, then the maximum,
+    // the weights and the denominator by shuffles; the partial rows are then fetched four splits at a time.
+    // Sums run over the splits in ascending order, as a plain loop would.
+    const float2* ml_row = part_ml + row * n_splits;
+    const float2 ml0 = lane < n_splits ? ml_row[lane] : make_float2(kNegInf, 0.f);
+    const float2 ml1 = lane + 32 < n_splits ? ml_row[lane + 32] : make_float2(kNegInf, 0.f);
+    float M = fmaxf(ml0.x, ml1.x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    const float w0 = ml0.y > 0.f ? expf(ml0.x - M) : 0.f;      // a split that saw no visible slot weighs nothing
+    const float w1 = ml1.y > 0.f ? expf(ml1.x - M) : 0.f;
     float L = 0.f, acc[kEpl];
 #pragma unroll
     for (int i = 0; i < kEpl; ++i) acc[i] = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-      const float2 ml = part_ml[row * n_splits + s];
-      if (ml.y <= 0.f) continue;
-      const float w = expf(ml.x - M);
-      L += ml.y * w;
-      const float* po = part_o + (row * n_splits + s) * kHeadDim + lane * kEpl;
+    const float* po_row = part_o + row * n_splits * kHeadDim + lane * kEpl;
+    for (int s0 = 0; s0 < n_splits; s0 += 4) {
+      float po[4][kEpl], w[4], lw[4];
 #pragma unroll
-      for (int i = 0; i < kEpl; ++i) acc[i] = fmaf(w, po[i], acc[i]);
+      for (int u = 0; u < 4; ++u) {
+        const int s = s0 + u;
+        const float ws = __shfl_sync(0xffffffffu, s < 32 ? w0 : w1, s & 31);
+        const float ls = __shfl_sync(0xffffffffu, s < 32 ? ml0.y : ml1.y, s & 31);
+        w[u] = s < n_splits ? ws : 0.f;
+        lw[u] = s < n_splits ? ls * ws : 0.f;
+        if (s < n_splits) {
+          if constexpr (kEpl == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(po_row + (size_t)s * kHeadDim);
+            po[u][0] = v.x; po[u][1] = v.y; po[u][2] = v.z; po[u][3] = v.w;
+          } else {
+            const float2 v = *reinterpret_cast<const float2*>(po_row + (size_t)s * kHeadDim);
+            po[u][0] = v.x; po[u][1] = v.y;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < kEpl; ++i) po[u][i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (w[u] > 0.f) {                                       // skipped splits may hold stale numbers, even NaN
+          L += lw[u];
+#pragma unroll
+          for (int i = 0; i < kEpl; ++i) acc[i] = fmaf(w[u], po[u][i], acc[i]);
+        }
+      }
     }
     const float inv = L > 0.f ? 1.0f / L : 0.f;
+    if constexpr (sizeof(T) == 2 && kEpl == 4) {
+      uint2 v;
+      v.x = ElemTraits<__nv_bfloat16>::pack2(acc[0] * inv, acc[1] * inv);
+      v.y = ElemTraits<__nv_bfloat16>::pack2(acc[2] * inv, acc[3] * inv);
+      *reinterpret_cast<uint2*>(O + row * kHeadDim + lane * kEpl) = v;
+    } else {
 #pragma unroll
-    for (int i = 0; i < kEpl; ++i) store_elem<T>(O + row * kHeadDim + lane * kEpl + i, acc[i] * inv);
+      for (int i = 0; i < kEpl; ++i) store_elem<T>(O + row * kHeadDim + lane * kEpl + i, acc[i] * inv);
+    }
     if (lse != nullptr && lane == 0) {
       const int hq = (int)(row % Hq);
       const long long bt = row / Hq;

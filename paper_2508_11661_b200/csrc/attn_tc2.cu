@@ -217,18 +217,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const int row_base = rtile * 2 * kBM;
   const int n_q = (rows_total - row_base > kBM) ? 2 : 1;      // query tiles that hold real rows
 
-  int len = cache_len[b];
-  len = max(0, min(len, capacity));
-  const int n_app = (appended && len + T_q <= capacity) ? T_q : 0;
-  const int total = len + n_app;
-  const int last_row = min(row_base + 2 * kBM, rows_total) - 1;
-  const int cta_visible = len + (n_app ? last_row / G + 1 : 0);
-  const int n_tiles = (total + kBN - 1) / kBN;
-  const int tps = (n_tiles + n_splits - 1) / n_splits;
-  const int tile0 = split * tps;
-  const int tile1 = min(min(tile0 + tps, n_tiles), (cta_visible + kBN - 1) / kBN);
-  const int nt = max(tile1 - tile0, 0);
-
   // ---- set-up ----
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) {
@@ -255,8 +243,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  // Q tiles: cp.async by the softmax warps (rows beyond the chunk zero-filled) while the loader already
-  // streams the first K/V tiles; the MMA thread waits for Q_READY before its first product
+  // Q tiles: cp.async by the softmax warps (rows beyond the chunk zero-filled); the MMA thread waits for Q_READY
+  // before its first product
   if (warp < kSoftmaxWarps) {
     for (int i = tid; i < 2 * kBM * 16; i += kSoftmaxWarps * 32) {
       const int r = i >> 4, c = i & 15;                       // r in [0, 256)
@@ -267,6 +255,25 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       cp_async16(sQ + (r >> 7) * kQBytes + (c >> 3) * (kBM * 128) + blk_off(r & 127, c & 7), src, ok);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+
+  // Everything above needs nothing from the kernel before this one in the stream (it may still be running when this
+  // kernel was launched as its programmatic dependent); everything below does: cache_len, the appended rows and the
+  // partial-result scratch.
+  pdl_wait();
+  int len = cache_len[b];
+  len = max(0, min(len, capacity));
+  const int n_app = (appended && len + T_q <= capacity) ? T_q : 0;
+  const int total = len + n_app;
+  const int last_row = min(row_base + 2 * kBM, rows_total) - 1;
+  const int cta_visible = len + (n_app ? last_row / G + 1 : 0);
+  const int n_tiles = (total + kBN - 1) / kBN;
+  const int tps = (n_tiles + n_splits - 1) / n_splits;
+  const int tile0 = split * tps;
+  const int tile1 = min(min(tile0 + tps, n_tiles), (cta_visible + kBN - 1) / kBN);
+  const int nt = max(tile1 - tile0, 0);
+
+  if (warp < kSoftmaxWarps) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     fence_proxy_async();
     __syncwarp();
@@ -275,7 +282,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
   if (warp == kLoadWarp) {
     // ================= loader: K ring and V ring =================
-    pdl_wait();                 // rows appended by the kernel before this one are in the cache from here on
     for (int j = 0; j < nt; ++j) {
       const int s = j % kStages;
       const uint32_t round = (uint32_t)(j / kStages);
