@@ -1,13 +1,13 @@
 // Per-context selection of SamKV (Sec. 3.2): protected initial/local units are always kept, the
 // middle units compete under a fixed budget.  One CTA per (layer, batch, kv head, context):
 // the middle scores are turned into order-preserving 32-bit keys held in shared memory, an
-// MSB-first radix select (4 passes of 8 bits) finds the k-th largest key, ties at that key are
+// MSB-first radix select (4 passes of 8 bits, two barriers each) finds the k-th largest key, ties at that key are
 // broken by index order with a block scan, and the kept ids are emitted already ascending.
 #include "common.cuh"
 
 namespace samkv {
 
-constexpr int kSelThreads = 256;
+constexpr int kSelThreads = 128;
 
 // float -> uint32 with the same ordering; -0 and +0 map to the same key.
 __device__ __forceinline__ uint32_t score_key(float x) {
@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int32_t* __restrict__ sel, const __grid_constant__ CtxTable ct,
               const __grid_constant__ SelTable st, int U_tot, int S_u, int* __restrict__ d_status) {
   extern __shared__ uint32_t keys[];         // [n_mid]
-  __shared__ uint32_t hist[256];
+  __shared__ uint32_t hist[4 * 256];         // one histogram per radix pass
   __shared__ uint32_t warp_tot[kSelThreads / 32];
   __shared__ uint32_t s_bin, s_remaining;
 
@@ -69,32 +69,47 @@ select_kernel(const float* __restrict__ scores, int32_t* __restrict__ sel, const
 
   const float* sc = scores + slab * U_tot + base + p0;
   for (int i = tid; i < n_mid; i += kSelThreads) keys[i] = score_key(sc[i]);
+  for (int i = tid; i < 4 * 256; i += kSelThreads) hist[i] = 0;
+  __syncthreads();
 
   // ---- radix select: the k_mid-th largest key ----
+  // One histogram per pass (all zeroed up front) and the bin search done by warp 0 alone with shuffles: two block
+  // barriers per pass.  The kernel is bound by barrier latency, not by bytes.
   uint32_t prefix = 0, mask = 0, remaining = (uint32_t)k_mid;
 #pragma unroll 1
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    hist[tid] = 0;
-    __syncthreads();   // also orders the key writes before the first pass
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    uint32_t* h = hist + pass * 256;
     for (int i = tid; i < n_mid; i += kSelThreads) {
       const uint32_t key = keys[i];
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      if ((key & mask) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    // count of candidates in bins above `tid`: total - inclusive prefix
-    const uint32_t mine = hist[tid];
-    uint32_t total;
-    const uint32_t below = block_exclusive_scan(mine, warp_tot, &total);
-    const uint32_t above = total - below - mine;
-    if (above < remaining && above + mine >= remaining) {   // exactly one bin satisfies this
-      s_bin = tid;
-      s_remaining = remaining - above;
+    if (tid < 32) {
+      // lane L owns bins [8L, 8L + 8); `above` = candidates in higher bins
+      uint32_t c[8], mine = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = h[tid * 8 + i]; mine += c[i]; }
+      uint32_t suffix = mine;                                   // inclusive sum over lanes >= this one
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_down_sync(0xffffffffu, suffix, o);
+        if (tid + o < 32) suffix += n;
+      }
+      uint32_t above = suffix - mine;
+#pragma unroll
+      for (int i = 7; i >= 0; --i) {
+        if (above < remaining && above + c[i] >= remaining) {   // exactly one bin of one lane satisfies this
+          s_bin = tid * 8 + i;
+          s_remaining = remaining - above;
+        }
+        above += c[i];
+      }
     }
     __syncthreads();
     prefix |= s_bin << shift;
     mask |= 255u << shift;
     remaining = s_remaining;
-    __syncthreads();
   }
   const uint32_t pivot = prefix;       // k-th largest key
   const uint32_t need_eq = remaining;  // how many keys equal to the pivot are kept (lowest indices first)
