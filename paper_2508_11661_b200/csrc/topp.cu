@@ -7,7 +7,9 @@
 
 namespace samkv {
 
-constexpr int kTopThreads = 256;
+constexpr int kTopThreads = 256;       // Top-P and the cross-context stage: few CTAs, many keys each
+constexpr int kRetrieveThreads = 128;  // per-document retrieval: many small CTAs, bound by per-CTA latency
+constexpr int kTopMaxWarps = kTopThreads / 32;
 
 __device__ __forceinline__ uint32_t order_key(float x) {      // float -> uint32, same ordering, -0 == +0
   uint32_t u = __float_as_uint(x);
@@ -20,12 +22,13 @@ __device__ __forceinline__ float key_to_float(uint32_t k) {
 
 // ---- block-wide helpers (kTopThreads threads) ------------------------------------------------------
 struct BlockScratch {
-  uint32_t hist[256];
-  uint32_t warp_tot[kTopThreads / 32];
-  float fred[3][kTopThreads / 32];
+  uint32_t hist[4 * 256];          // one histogram per radix pass
+  uint32_t warp_tot[kTopMaxWarps];
+  float fred[3][kTopMaxWarps];
   uint32_t bin, remaining;
 };
 
+template <int kT>
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, BlockScratch& sc, uint32_t* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t inc = v;
@@ -39,7 +42,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, BlockScratch& sc
   __syncthreads();
   uint32_t before = 0, tot = 0;
 #pragma unroll
-  for (int i = 0; i < kTopThreads / 32; ++i) {
+  for (int i = 0; i < kT / 32; ++i) {
     const uint32_t t = sc.warp_tot[i];
     if (i < warp) before += t;
     tot += t;
@@ -49,6 +52,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, BlockScratch& sc
 }
 
 // (sum, max, min) over the block in a fixed order
+template <int kT>
 __device__ __forceinline__ void block_reduce3(float& s, float& mx, float& mn, BlockScratch& sc) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -61,7 +65,7 @@ __device__ __forceinline__ void block_reduce3(float& s, float& mx, float& mn, Bl
   if (lane == 0) { sc.fred[0][warp] = s; sc.fred[1][warp] = mx; sc.fred[2][warp] = mn; }
   __syncthreads();
   s = 0.f; mx = -INFINITY; mn = INFINITY;
-  for (int i = 0; i < kTopThreads / 32; ++i) {
+  for (int i = 0; i < kT / 32; ++i) {
     s += sc.fred[0][i];
     mx = fmaxf(mx, sc.fred[1][i]);
     mn = fminf(mn, sc.fred[2][i]);
@@ -70,29 +74,45 @@ __device__ __forceinline__ void block_reduce3(float& s, float& mx, float& mn, Bl
 
 // k-th largest of the non-zero keys keys[0..n) (zero marks "not a candidate"); 1 <= k <= number of candidates.
 // Returns the pivot key and how many keys equal to it belong to the top k (lowest indices first).
+// MSB-first radix select, 4 passes of 8 bits: one histogram per pass (zeroed up front), the bin search by warp 0
+// with shuffles, two block barriers per pass.
+template <int kT>
 __device__ __forceinline__ void block_radix_select(const uint32_t* keys, int n, uint32_t k, BlockScratch& sc,
                                                    uint32_t* pivot, uint32_t* need_eq) {
   const int tid = threadIdx.x;
+  for (int i = tid; i < 4 * 256; i += kT) sc.hist[i] = 0;
+  __syncthreads();
   uint32_t prefix = 0, mask = 0, remaining = k;
 #pragma unroll 1
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    sc.hist[tid] = 0;
-    __syncthreads();
-    for (int i = tid; i < n; i += kTopThreads) {
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    uint32_t* h = sc.hist + pass * 256;
+    for (int i = tid; i < n; i += kT) {
       const uint32_t key = keys[i];
-      if (key != 0 && (key & mask) == prefix) atomicAdd(&sc.hist[(key >> shift) & 255u], 1u);
+      if (key != 0 && (key & mask) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    const uint32_t mine = sc.hist[tid];
-    uint32_t total;
-    const uint32_t below = block_excl_scan(mine, sc, &total);
-    const uint32_t above = total - below - mine;
-    if (above < remaining && above + mine >= remaining) { sc.bin = tid; sc.remaining = remaining - above; }
+    if (tid < 32) {
+      uint32_t c[8], mine = 0;                                   // lane L owns bins [8L, 8L + 8)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = h[tid * 8 + i]; mine += c[i]; }
+      uint32_t suffix = mine;                                    // inclusive sum over lanes >= this one
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, suffix, o);
+        if (tid + o < 32) suffix += v;
+      }
+      uint32_t above = suffix - mine;
+#pragma unroll
+      for (int i = 7; i >= 0; --i) {
+        if (above < remaining && above + c[i] >= remaining) { sc.bin = tid * 8 + i; sc.remaining = remaining - above; }
+        above += c[i];
+      }
+    }
     __syncthreads();
     prefix |= sc.bin << shift;
     mask |= 255u << shift;
     remaining = sc.remaining;
-    __syncthreads();
   }
   *pivot = prefix;
   *need_eq = remaining;
@@ -144,7 +164,7 @@ topp_kernel(const float* __restrict__ scores, const int32_t* __restrict__ max_un
           mn = fminf(mn, v);
         }
       }
-      block_reduce3(anc, mx, mn, sc);
+      block_reduce3<kTopThreads>(anc, mx, mn, sc);
       if (p1 > p0) {
         const int n_prot_tok = min(p0 * B, L_c) + (L_c - min(p1 * B, L_c));
         const float s_anc = n_prot_tok > 0 ? anc / (float)n_prot_tok : 0.f;
@@ -172,7 +192,7 @@ topp_kernel(const float* __restrict__ scores, const int32_t* __restrict__ max_un
 // units of the context (ties: lower index) and append them, ascending by unit id, to the slab's candidate list
 // at cand_off[c]: ckey = order key of the min-max normalised score (never 0), cid = global unit id.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTopThreads)
+__global__ void __launch_bounds__(kRetrieveThreads)
 retrieve_kernel(const float* __restrict__ scores, uint32_t* __restrict__ ckey, int32_t* __restrict__ cid,
                 const __grid_constant__ CtxTable ct, const __grid_constant__ TopTable tt, int U_tot, int C_tot) {
   extern __shared__ uint32_t kc[];                              // [n_mid] order keys of the middle units' scores
@@ -186,17 +206,17 @@ retrieve_kernel(const float* __restrict__ scores, uint32_t* __restrict__ ckey, i
   if (n_mid <= 0 || want <= 0) return;
   const float* u = scores + slab * U_tot + base + p0;
   float dummy = 0.f, hi = -INFINITY, lo = INFINITY;
-  for (int i = tid; i < n_mid; i += kTopThreads) {
+  for (int i = tid; i < n_mid; i += kRetrieveThreads) {
     const float v = u[i];
     kc[i] = order_key(v);
     hi = fmaxf(hi, v);
     lo = fminf(lo, v);
   }
-  block_reduce3(dummy, hi, lo, sc);                             // its barriers also publish kc to the block
+  block_reduce3<kRetrieveThreads>(dummy, hi, lo, sc);                             // its barriers also publish kc to the block
   uint32_t pivot = 0, need_eq = 0xffffffffu;                    // want == n_mid: every key is above the pivot
-  if (want < n_mid) block_radix_select(kc, n_mid, (uint32_t)want, sc, &pivot, &need_eq);
+  if (want < n_mid) block_radix_select<kRetrieveThreads>(kc, n_mid, (uint32_t)want, sc, &pivot, &need_eq);
   // ordered pass: keys above the pivot, and the first need_eq keys equal to it, in ascending unit order
-  const int per = (n_mid + kTopThreads - 1) / kTopThreads;
+  const int per = (n_mid + kRetrieveThreads - 1) / kRetrieveThreads;
   const int a = min(tid * per, n_mid), e = min(a + per, n_mid);
   uint32_t gt = 0, eq = 0;
   for (int i = a; i < e; ++i) {
@@ -204,7 +224,7 @@ retrieve_kernel(const float* __restrict__ scores, uint32_t* __restrict__ ckey, i
     eq += (kc[i] == pivot);
   }
   uint32_t total;
-  const uint32_t packed = block_excl_scan((gt << 16) | eq, sc, &total);      // both counts < 2^16 (units per context)
+  const uint32_t packed = block_excl_scan<kRetrieveThreads>((gt << 16) | eq, sc, &total);      // both counts < 2^16 (units per context)
   uint32_t gt_before = packed >> 16, eq_before = packed & 0xffffu;
   const float range = hi - lo;
   uint32_t* dkey = ckey + slab * C_tot + tt.cand_off[c];
@@ -243,12 +263,12 @@ cross_topk_kernel(const uint32_t* __restrict__ ckey_all, const int32_t* __restri
   int32_t* out = sel + slab * S_u;
   const int tid = threadIdx.x;
   const int D = ct.n_ctx;
-  if (tid <= SAMKV_MAX_CTX) s_chosen[tid] = 0;
+  for (int i = tid; i <= SAMKV_MAX_CTX; i += kTopThreads) s_chosen[i] = 0;
   __syncthreads();
 
   if (K > 0) {
     uint32_t pivot = 0, need_eq = 0xffffffffu;                  // K == C_tot: everything retrieved is kept
-    if (K < C_tot) block_radix_select(ckey, C_tot, (uint32_t)K, sc, &pivot, &need_eq);
+    if (K < C_tot) block_radix_select<kTopThreads>(ckey, C_tot, (uint32_t)K, sc, &pivot, &need_eq);
     const int per = (C_tot + kTopThreads - 1) / kTopThreads;
     const int a = min(tid * per, C_tot), e = min(a + per, C_tot);
     uint32_t gt = 0, eq = 0;
@@ -257,8 +277,8 @@ cross_topk_kernel(const uint32_t* __restrict__ ckey_all, const int32_t* __restri
       eq += (ckey[i] == pivot);
     }
     uint32_t total;
-    uint32_t gt_before = block_excl_scan(gt, sc, &total);
-    uint32_t eq_before = block_excl_scan(eq, sc, &total);
+    uint32_t gt_before = block_excl_scan<kTopThreads>(gt, sc, &total);
+    uint32_t eq_before = block_excl_scan<kTopThreads>(eq, sc, &total);
     int c = (a < e) ? find_segment(tt.cand_off, D, a) : 0;
     for (int i = a; i < e; ++i) {
       while (i >= tt.cand_off[c + 1]) ++c;
@@ -394,7 +414,7 @@ cudaError_t launch_select_cross(const samkv_shape_t& s, const CtxTable& ct, cons
       cudaError_t e = cudaFuncSetAttribute(retrieve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
-    retrieve_kernel<<<(unsigned)(slabs * ct.n_ctx), kTopThreads, smem, stream>>>(scores, ckey, cid, ct, tt, U_tot, C_tot);
+    retrieve_kernel<<<(unsigned)(slabs * ct.n_ctx), kRetrieveThreads, smem, stream>>>(scores, ckey, cid, ct, tt, U_tot, C_tot);
   }
   cross_topk_kernel<<<(unsigned)slabs, kTopThreads, 0, stream>>>(ckey, cid, sel, counts, ct, tt, C_tot, S_u, K);
   return cudaGetLastError();
