@@ -326,3 +326,40 @@ def test_context_beyond_shared_memory_is_refused():
     with pytest.raises(B.SamkvError) as e:
         B.samkv_budget_units(shape, 1500)                               # more units in one context than the select kernel holds
     assert e.value.status == 2
+
+
+def test_chunked_prefill_on_the_tensor_memory_kernel():
+    """Three consecutive 64-token chunks on the same layer (256 packed rows per KV head, so every call takes the
+    tcgen05 kernel and its dependent-launch chain: append -> attention -> merge).  Each call must see the cache
+    length and the rows the previous call left, then a cache-only call must see all three chunks."""
+    w = synth.CONFIGS["cfg1"].replace(name="cfg1_chunks", batch=2, q_tokens=64, ctx_lens=(1024, 700, 1300))
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = GpuRun(w, inp, extra_capacity=3 * 64).sparsify()
+    torch.cuda.synchronize()
+    Kc_ref = [to_f64(run.Kc[0, b]) for b in range(w.batch)]
+    Vc_ref = [to_f64(run.Vc[0, b]) for b in range(w.batch)]
+    n = run.S
+    g = torch.Generator().manual_seed(17)
+    outs = []
+    for chunk in range(3):                                      # launched back to back, no host synchronisation
+        q = torch.randn((w.batch, 64, w.n_q_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        kq = torch.randn((w.batch, 64, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        vq = torch.randn((w.batch, 64, w.n_kv_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+        outs.append((q, kq, vq) + run.attn(0, q, kq, vq))
+    q_last = torch.randn((w.batch, 64, w.n_q_heads, w.head_dim), generator=g).to(w.torch_dtype).to(DEV)
+    O_last, lse_last = run.attn(0, q_last)                      # cache only, right behind an appending call
+    torch.cuda.synchronize()
+    assert run.poll() == 0
+    for q, kq, vq, Os, ls in outs:
+        for b in range(w.batch):
+            out, l2, Kc_ref[b], Vc_ref[b], n2 = O.attention(Kc_ref[b], Vc_ref[b], n, to_f64(q[b]), to_f64(kq[b]),
+                                                            to_f64(vq[b]))
+            assert np.abs(to_f64(Os[b]) - out).max() <= 2e-2
+            assert np.abs(to_f64(ls[b]) - l2).max() <= 2e-2
+        n += 64
+    assert run.cache_len.cpu().tolist() == [[n] * w.batch]
+    for b in range(w.batch):
+        out, l2, _, _, _ = O.attention(Kc_ref[b], Vc_ref[b], n, to_f64(q_last[b]))
+        assert np.abs(to_f64(O_last[b]) - out).max() <= 2e-2
+        assert np.abs(to_f64(lse_last[b]) - l2).max() <= 2e-2
+        assert np.array_equal(to_f64(run.Kc[0, b])[:, :n], Kc_ref[b][:, :n])
