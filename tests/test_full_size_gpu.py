@@ -151,3 +151,36 @@ def test_cfg4_stress_budget_sweep(budget_bp):
     assert int(run.cache_len[0, 0]) == run.S + w.q_tokens and run.poll() == 0
     del run, inp
     _free_all()
+
+
+def test_cfg2_timed_schedule_matches_in_order_and_oracle():
+    """The schedule bench.py times (scoring + selection of all layers, then 8 layer groups whose gather + update
+    overlap the attention of earlier groups on a second stream, per-layer attention calls through a second handle)
+    must give bit-identical results to the same calls issued in order on one stream, and its attention output
+    must match the oracle on sampled (layer, batch element) problems."""
+    import bench
+    w = synth.CONFIGS["cfg2"]
+    pipe = bench.Pipeline(w, torch.device(DEV))
+    pipe.prepare_recompute()
+    assert pipe.groups == 8 and pipe.R == 690
+    pipe.step(overlap=False)
+    torch.cuda.synchronize()
+    ref = {"O": pipe.O.clone(), "sel": pipe.sel.clone(), "cache_len": pipe.cache_len.clone(),
+           "Kc": pipe.Kc[::7].clone(), "Vc": pipe.Vc[::7].clone(), "scores": pipe.scores[::7].clone()}
+    pipe.O.zero_(); pipe.sel.zero_(); pipe.cache_len.zero_(); pipe.Kc.zero_(); pipe.Vc.zero_(); pipe.scores.zero_()
+    for _ in range(2):                                   # twice: the second pass starts from the first one's state
+        pipe.step(overlap=True)
+    torch.cuda.synchronize()
+    assert B.samkv_poll_status(pipe.handle) == 0 and B.samkv_poll_status(pipe.handle_attn) == 0
+    assert torch.equal(pipe.sel, ref["sel"]) and torch.equal(pipe.cache_len, ref["cache_len"])
+    assert torch.equal(pipe.scores[::7], ref["scores"])
+    assert torch.equal(pipe.Kc[::7].view(torch.int16), ref["Kc"].view(torch.int16))
+    assert torch.equal(pipe.Vc[::7].view(torch.int16), ref["Vc"].view(torch.int16))
+    assert torch.equal(pipe.O.view(torch.int16), ref["O"].view(torch.int16))
+    assert int(pipe.cache_len[0, 0]) == pipe.S + w.q_tokens
+    inp = pipe.inp
+    for (l, b) in [(0, 0), (13, 1), (31, 3)]:
+        check_attention(w, pipe.Kc[l, b], pipe.Vc[l, b], pipe.S, inp["Qa"][l, b], inp["Kq"][l, b], inp["Vq"][l, b],
+                        pipe.O[l, b])
+    del pipe, ref
+    _free_all()
