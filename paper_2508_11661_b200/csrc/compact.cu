@@ -134,6 +134,13 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
   bool active = row < n_rows;
   int slot = -1;
   size_t slab = 0;
+  // the new rows depend on nothing but the row index: fetch them while the token -> slot look-ups are in flight
+  uint4 kn = make_uint4(0, 0, 0, 0), vn = kn, ko = kn, vo = kn;
+  if (active) {
+    const size_t src = (size_t)row * kHeadDim + lane * kPerVec;
+    kn = ld_stream(Knew + src);
+    vn = ld_stream(Vnew + src);
+  }
   if (active) {
     const int h = (int)(row % Hkv);
     const long long lbr = row / Hkv;
@@ -146,13 +153,9 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
     if (slot >= capacity) slot = -1;
   }
   active = slot >= 0;
-  uint4 kn = make_uint4(0, 0, 0, 0), vn = kn, ko = kn, vo = kn;
   size_t dst = 0;
   if (active) {
-    const size_t src = (size_t)row * kHeadDim + lane * kPerVec;
     dst = (slab * capacity + slot) * kHeadDim + lane * kPerVec;
-    kn = ld_stream(Knew + src);
-    vn = ld_stream(Vnew + src);
     if (mode == SAMKV_UPDATE_FUSION) {
       ko = *reinterpret_cast<const uint4*>(Kc + dst);
       vo = *reinterpret_cast<const uint4*>(Vc + dst);
