@@ -27,12 +27,12 @@ compact_kernel(const char* __restrict__ K, const char* __restrict__ V, const int
 
   if (chunk == 0 && threadIdx.x == 0 && (slab % Hkv) == 0) cache_len[slab / Hkv] = S;
 
-  uint4 kv[kPasses], vv[kPasses];
-  int tok[kPasses];
-#pragma unroll
-  for (int p = 0; p < kPasses; ++p) {
-    const int slot = chunk * kCompactRowsPerCta + p * kRowsPerPass + rsub;
-    tok[p] = -1;
+  // slot -> source token, once per slot of the CTA (one thread each) instead of once per 16-byte lane: the search
+  // over the context table and the dependent read of the unit list leave the copy loop
+  __shared__ int s_tok[kCompactRowsPerCta];
+  if (threadIdx.x < kCompactRowsPerCta) {
+    const int slot = chunk * kCompactRowsPerCta + threadIdx.x;
+    int t = -1;
     if (slot < S) {
       const int c = find_segment(st.slot_off, ct.n_ctx, slot);
       const int r = slot - st.slot_off[c];
@@ -40,15 +40,25 @@ compact_kernel(const char* __restrict__ K, const char* __restrict__ V, const int
       // without a list (sel == nullptr) the kept units are the protected ones: two contiguous ranges per context
       const int m = sel != nullptr ? sel[slab * S_u + st.sel_off[c] + j] - ct.unit_off[c]
                                    : (j < st.n_init_units[c] ? j : st.first_local_unit[c] + (j - st.n_init_units[c]));
-      const int t = ct.ctx_off[c] + (m << ct.block_shift) + (r & (ct.block_size - 1));
+      t = ct.ctx_off[c] + (m << ct.block_shift) + (r & (ct.block_size - 1));
       if (m < 0 || m >= ct.unit_off[c + 1] - ct.unit_off[c] || t >= ct.ctx_off[c + 1]) {
-        if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);
-      } else {
-        tok[p] = t;
-        const size_t src = (slab * L_tot + t) * kRowBytes + lane * 16;
-        kv[p] = *reinterpret_cast<const uint4*>(K + src);
-        vv[p] = ld_stream(V + src);
+        atomicMax(d_status, (int)CHECK_SEL_RANGE);
+        t = -1;
       }
+    }
+    s_tok[threadIdx.x] = t;
+  }
+  __syncthreads();
+
+  uint4 kv[kPasses], vv[kPasses];
+  int tok[kPasses];
+#pragma unroll
+  for (int p = 0; p < kPasses; ++p) {
+    tok[p] = s_tok[p * kRowsPerPass + rsub];
+    if (tok[p] >= 0) {
+      const size_t src = (slab * L_tot + tok[p]) * kRowBytes + lane * 16;
+      kv[p] = *reinterpret_cast<const uint4*>(K + src);
+      vv[p] = ld_stream(V + src);
     }
   }
 #pragma unroll
@@ -128,10 +138,13 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
   constexpr int kLanes = kHeadDim / kPerVec;
   constexpr int kRowsPerCta = kCopyThreads / kLanes;
   const int lane = threadIdx.x % kLanes;
-  const long long row = (long long)blockIdx.x * kRowsPerCta + threadIdx.x / kLanes;   // ((l*Bt + b)*R + r)*Hkv + h
+  // blockIdx.y = l*Bt + b; blockIdx.x walks the R*Hkv rows of that (layer, batch element) in 32-bit arithmetic
+  const int lb = blockIdx.y;
+  const int rh = blockIdx.x * kRowsPerCta + threadIdx.x / kLanes;                      // r*Hkv + h
+  const long long row = (long long)lb * (R * Hkv) + rh;                                // ((l*Bt + b)*R + r)*Hkv + h
   // Whole kLanes-groups take the same branch, and kLanes divides 32, so shuffles inside fuse_vec are
   // executed by complete groups; inactive groups are masked out below without leaving the warp.
-  bool active = row < n_rows;
+  bool active = rh < R * Hkv && row < n_rows;
   int slot = -1;
   size_t slab = 0;
   // the new rows depend on nothing but the row index: fetch them while the token -> slot look-ups are in flight
@@ -142,12 +155,9 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
     vn = ld_stream(Vnew + src);
   }
   if (active) {
-    const int h = (int)(row % Hkv);
-    const long long lbr = row / Hkv;
-    const int r = (int)(lbr % R);
-    const long long lb = lbr / R;
-    const long long l = lb / Bt;
-    const int t = tok_ids[l * R + r];
+    const int r = rh / Hkv, h = rh - r * Hkv;
+    const int l = lb / Bt;
+    const int t = tok_ids[(size_t)l * R + r];
     slab = (size_t)lb * Hkv + h;
     if (t >= 0 && t < L_tot) slot = inv_map[slab * L_tot + t];
     if (slot >= capacity) slot = -1;
@@ -179,9 +189,10 @@ cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc,
 #define SAMKV_LAUNCH_UPDATE(T, HD)                                                                                 \
   do {                                                                                                             \
     constexpr int rows_per_cta = kCopyThreads / (HD / ElemTraits<T>::kPerVec);                                     \
-    const long long blocks = (n_rows + rows_per_cta - 1) / rows_per_cta;                                           \
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;                                               \
-    update_kernel<T, HD><<<(unsigned)blocks, kCopyThreads, 0, stream>>>((T*)Kc, (T*)Vc, inv_map, tok_ids,           \
+    const long long per_lb = ((long long)R * s.n_kv_heads + rows_per_cta - 1) / rows_per_cta;                      \
+    const long long n_lb = (long long)s.n_layers * s.batch;                                                        \
+    if (per_lb > 0x7fffffffLL || n_lb > 65535) return cudaErrorInvalidConfiguration;                               \
+    update_kernel<T, HD><<<dim3((unsigned)per_lb, (unsigned)n_lb), kCopyThreads, 0, stream>>>((T*)Kc, (T*)Vc, inv_map, tok_ids, \
                                                                        (const T*)Knew, (const T*)Vnew, s.batch,    \
                                                                        s.n_kv_heads, R, L_tot, capacity, mode,     \
                                                                        n_rows);                                    \
