@@ -334,29 +334,52 @@ compact_units_kernel(const char* __restrict__ K, const char* __restrict__ V, con
   const int lane = threadIdx.x % kLanes, rsub = threadIdx.x / kLanes;
   if (chunk == 0 && threadIdx.x == 0 && (slab % Hkv) == 0) cache_len[slab / Hkv] = S;
   const int B = ct.block_size;
+  // virtual row (list position * B + offset in unit) -> (source token, slot), once per row of the CTA
+  __shared__ int s_tok[64], s_slot[64];
+  if (threadIdx.x < 64) {
+    const int v = chunk * 64 + threadIdx.x;
+    int t = -1, slot = -1;
+    if (v < S_u * B) {
+      const int pos = v >> ct.block_shift, j = v & (B - 1);
+      const int unit = sel[slab * S_u + pos];
+      if (unit < 0 || unit >= ct.unit_off[ct.n_ctx]) {
+        atomicMax(d_status, (int)CHECK_SEL_RANGE);
+      } else {
+        const int c = find_segment(ct.unit_off, ct.n_ctx, unit);
+        t = ct.ctx_off[c] + ((unit - ct.unit_off[c]) << ct.block_shift) + j;
+        slot = pos * B - tt.deficit_before[c] + j;
+        if (t >= ct.ctx_off[c + 1]) {
+          t = -1;                                                   // beyond the end of a short tail unit
+        } else if (slot < 0 || slot >= S) {
+          atomicMax(d_status, (int)CHECK_SEL_RANGE);                // the list is not what samkv_select_cross writes
+          t = -1;
+        }
+      }
+    }
+    s_tok[threadIdx.x] = t;
+    s_slot[threadIdx.x] = slot;
+  }
+  __syncthreads();
+  uint4 kv[kPasses], vv[kPasses];
+  int tok[kPasses];
 #pragma unroll
   for (int p = 0; p < kPasses; ++p) {
-    const int v = chunk * 64 + p * kRowsPerPass + rsub;          // virtual row: list position * B + offset in unit
-    if (v >= S_u * B) continue;
-    const int pos = v >> ct.block_shift, j = v & (B - 1);
-    const int unit = sel[slab * S_u + pos];
-    if (unit < 0 || unit >= ct.unit_off[ct.n_ctx]) {
-      if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);
-      continue;
+    tok[p] = s_tok[p * kRowsPerPass + rsub];
+    if (tok[p] >= 0) {
+      const size_t src = (slab * L_tot + tok[p]) * kRowBytes + lane * 16;
+      kv[p] = *reinterpret_cast<const uint4*>(K + src);
+      vv[p] = ld_stream(V + src);
     }
-    const int c = find_segment(ct.unit_off, ct.n_ctx, unit);
-    const int t = ct.ctx_off[c] + ((unit - ct.unit_off[c]) << ct.block_shift) + j;
-    if (t >= ct.ctx_off[c + 1]) continue;                          // beyond the end of a short tail unit
-    const int slot = pos * B - tt.deficit_before[c] + j;
-    if (slot < 0 || slot >= S) {
-      if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);   // the list is not what samkv_select_cross writes
-      continue;
+  }
+#pragma unroll
+  for (int p = 0; p < kPasses; ++p) {
+    if (tok[p] >= 0) {
+      const int slot = s_slot[p * kRowsPerPass + rsub];
+      const size_t dst = (slab * capacity + slot) * kRowBytes + lane * 16;
+      *reinterpret_cast<uint4*>(Kc + dst) = kv[p];
+      *reinterpret_cast<uint4*>(Vc + dst) = vv[p];
+      if (inv_map != nullptr && lane == 0) inv_map[slab * L_tot + tok[p]] = slot;
     }
-    const size_t src = (slab * L_tot + t) * kRowBytes + lane * 16;
-    const size_t dst = (slab * capacity + slot) * kRowBytes + lane * 16;
-    *reinterpret_cast<uint4*>(Kc + dst) = *reinterpret_cast<const uint4*>(K + src);
-    *reinterpret_cast<uint4*>(Vc + dst) = ld_stream(V + src);
-    if (inv_map != nullptr && lane == 0) inv_map[slab * L_tot + t] = slot;
   }
 }
 
