@@ -23,47 +23,63 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
                             cudaStream_t stream);
+cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
+                            const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
+                            float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
+                            cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Plan: how many packed rows a CTA takes and into how many KV splits a (batch, kv head) is cut.
 // The host does not know cache_len (it lives on the device), so splits are sized from capacity.
 // ---------------------------------------------------------------------------------------------
-AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) {
-  AttnPlan p;
-  const int G = s.n_q_heads / s.n_kv_heads;
-  const int rows = T_q * G;
-  int ctas_per_sm, slots_per_tile, min_slots;
-  if (s.dtype == SAMKV_BF16) {
-    // >= 128 packed rows and d = 128: the warp-specialised tcgen05 kernel (two 128-row tiles per CTA, one CTA
-    // per SM); otherwise mma.sync with 64 or 16 rows per CTA
-    const bool tc = rows >= 128 && s.head_dim == 128;
-    p.rows_per_cta = tc ? 256 : (rows > 16 ? 64 : 16);
-    ctas_per_sm = tc ? 1 : (rows > 16 ? 2 : 3);   // shared memory / registers of the attention kernels
-    slots_per_tile = tc ? 128 : 64;
-    min_slots = 256;
-  } else {
-    p.rows_per_cta = kSimtWarps;
-    ctas_per_sm = 8;
-    slots_per_tile = 64;
-    min_slots = 64;
-  }
-  const long long row_tiles = (rows + p.rows_per_cta - 1) / p.rows_per_cta;
-  const long long base_ctas = (long long)s.batch * s.n_kv_heads * row_tiles;
-  long long max_splits = capacity / min_slots;
-  if (max_splits > 64) max_splits = 64;
-  if (max_splits < 1) max_splits = 1;
-  // Pick the split count with the least (waves x work per CTA): a grid that spills a few CTAs into one
-  // more wave costs a whole wave, and every CTA pays a fixed prologue/epilogue (taken as 3 tiles).
-  const long long tiles = (capacity + slots_per_tile - 1) / slots_per_tile;
-  const long long slots = (long long)sm_count * ctas_per_sm;
+// Best split count for one kernel shape: least (waves x time per CTA), where a CTA costs `tile_cost` per KV tile
+// plus `fixed_cost` for its prologue and epilogue (any common unit).  A grid that spills a few CTAs into one more
+// wave costs a whole wave.
+static long long best_split(long long base_ctas, long long tiles, long long slots, long long max_splits,
+                            long long tile_cost, long long fixed_cost, long long* cost_out) {
   long long best_n = 1, best_cost = -1;
   for (long long n = 1; n <= max_splits; ++n) {
     const long long tps = (tiles + n - 1) / n;
     const long long waves = (base_ctas * n + slots - 1) / slots;
-    const long long cost = waves * (tps + 3);
+    const long long cost = waves * (tps * tile_cost + fixed_cost);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
   }
-  p.n_splits = (int)best_n;
+  *cost_out = best_cost;
+  return best_n;
+}
+
+AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) {
+  AttnPlan p;
+  const int G = s.n_q_heads / s.n_kv_heads;
+  const int rows = T_q * G;
+  const long long bh = (long long)s.batch * s.n_kv_heads;
+  const long long min_slots = s.dtype == SAMKV_BF16 ? 256 : 64;
+  long long max_splits = capacity / min_slots;
+  if (max_splits > 64) max_splits = 64;
+  if (max_splits < 1) max_splits = 1;
+  long long cost = 0;
+  if (s.dtype == SAMKV_BF16 && rows >= 128 && s.head_dim == 128) {
+    // The two tcgen05 kernels, one CTA per SM, 128-slot tiles.  Measured on B200 (cycles): 256 rows per CTA
+    // (two query tiles share every K/V tile) ~5000 per tile + ~20000 per CTA; 128 rows per CTA (score tile
+    // double-buffered) ~2760 per tile + ~9000 per CTA.  Short KV ranges favour the second, long ones the first.
+    const long long tiles = (capacity + 127) / 128;
+    long long cost256 = 0, cost128 = 0;
+    const long long n256 = best_split(bh * ((rows + 255) / 256), tiles, sm_count, max_splits, 5000, 20000, &cost256);
+    const long long n128 = best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2760, 9000, &cost128);
+    const bool use128 = cost128 <= cost256;
+    p.rows_per_cta = use128 ? 128 : 256;
+    p.n_splits = (int)(use128 ? n128 : n256);
+  } else if (s.dtype == SAMKV_BF16) {
+    // mma.sync kernel with 64 or 16 rows per CTA, 64-slot tiles; the fixed part is taken as 3 tiles
+    p.rows_per_cta = rows > 16 ? 64 : 16;
+    const long long ctas_per_sm = rows > 16 ? 2 : 3;          // shared memory / registers of the kernel
+    p.n_splits = (int)best_split(bh * ((rows + p.rows_per_cta - 1) / p.rows_per_cta), (capacity + 63) / 64,
+                                 sm_count * ctas_per_sm, max_splits, 1, 3, &cost);
+  } else {
+    p.rows_per_cta = kSimtWarps;
+    p.n_splits = (int)best_split(bh * ((rows + kSimtWarps - 1) / kSimtWarps), (capacity + 63) / 64,
+                                 (long long)sm_count * 8, max_splits, 1, 3, &cost);
+  }
   const size_t out_rows = (size_t)s.batch * T_q * s.n_q_heads;
   p.partial_bytes = p.n_splits > 1 ? out_rows * p.n_splits * ((size_t)s.head_dim * 4 + 8) : 0;
   return p;
@@ -311,7 +327,10 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int G = Hq / Hkv;
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
-    cudaError_t e = (plan.rows_per_cta == 256)
+    cudaError_t e = (plan.rows_per_cta == 128)
+                        ? launch_attn_tc3(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                                          plan, d_status, stream)
+                    : (plan.rows_per_cta == 256)
                         ? launch_attn_tc2(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
                                           plan, d_status, stream)
                         : launch_attn_mma(s, layer, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o,
@@ -334,7 +353,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
-    if (sizeof(T) == 2 && plan.rows_per_cta == 256) {     // the tensor-memory kernel releases its dependents early
+    if (sizeof(T) == 2 && plan.rows_per_cta >= 128) {     // the tensor-memory kernels release their dependents early
       cfg.attrs = &attr;
       cfg.numAttrs = 1;
     }
