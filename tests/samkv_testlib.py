@@ -19,7 +19,7 @@ def oracle_k_units(w) -> list:
     return [O.budget_units(n, w.block_size, w.n_init, w.n_local, w.budget_bp) for n in w.ctx_lens]
 
 
-class GpuRun:
+class DeviceRun:
     """One pass of the library over a workload; keeps every intermediate tensor."""
 
     def __init__(self, w, inp, k_units=None, use_bias=True, extra_capacity=None, with_qloc=True):
@@ -86,7 +86,7 @@ def oracle_scores(w, inp, l, b, use_bias=True, with_qloc=True):
     return q, s, u
 
 
-def check_scores(w, run: GpuRun, l, b, q, u, K64=None):
+def check_scores(w, run: DeviceRun, l, b, q, u, K64=None):
     """Scores and q^ are diagnostics: |gpu - oracle| <= 1e-5 * ||q|| * ||K row|| (bounded here by the
     largest row norm of the slab), q^ to 1e-5 relative to its norm."""
     qg = run.qhat[l, b].cpu().double().numpy()                           # [D, Hkv, d]
@@ -136,7 +136,7 @@ def check_selection(w, k_units, sel_gpu_lb: np.ndarray, u: np.ndarray, where="")
     return n_diff
 
 
-def check_compact(w, run: GpuRun, l, b, sel_lb: np.ndarray):
+def check_compact(w, run: DeviceRun, l, b, sel_lb: np.ndarray):
     """Bit-exact gather with the GPU's own index set; inverse map round trip; cache_len."""
     K = run.inp["K"][l, b].cpu()
     V = run.inp["V"][l, b].cpu()

@@ -9,7 +9,7 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import GpuRun
+from samkv_testlib import DeviceRun
 
 pytestmark = pytest.mark.gpu
 
@@ -53,7 +53,7 @@ def random_inv_map(L, Bt, Hkv, L_tot, p, seed, device="cuda"):
 def small_run(L=4, Bt=2, ctx_lens=(300, 257, 130), seed=7):
     w = dataclasses.replace(synth.ragged_workload(ctx_lens=ctx_lens, seed=seed), n_layers=L, batch=Bt)
     inp = synth.make_inputs(w, "cuda")
-    return w, GpuRun(w, inp)
+    return w, DeviceRun(w, inp)
 
 
 def test_align_after_fixed_budget_selection():
@@ -80,7 +80,7 @@ def test_align_after_fixed_budget_selection():
 def test_align_random_maps(L, Bt, Hkv, p, seed):
     w = dataclasses.replace(synth.ragged_workload(ctx_lens=(211, 190), n_q_heads=Hkv * 2, n_kv_heads=Hkv, seed=seed),
                             n_layers=L, batch=Bt)
-    run = GpuRun(w, synth.make_inputs(w, "cuda"))
+    run = DeviceRun(w, synth.make_inputs(w, "cuda"))
     inv = random_inv_map(L, Bt, Hkv, w.l_tot, p, seed)
     g = torch.Generator().manual_seed(seed)
     tok = torch.stack([torch.randperm(w.l_tot, generator=g)[:25] for _ in range(L)]).to(torch.int32).cuda()
@@ -115,7 +115,7 @@ def test_align_bench_shape_sample():
     """cfg2's token axis (30 720 tokens, 8 heads) on 4 layers; the oracle checks one batch element."""
     w = dataclasses.replace(synth.CONFIGS["cfg2"], name="align_cfg2", n_layers=4, batch=2)
     inp = synth.make_inputs(w, "cuda")
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     sel_tok = torch.stack([torch.nonzero(run.inv_map[n, 0, 0] >= 0).flatten() for n in range(w.n_layers)])
     tok, _, _ = synth.make_recompute(w, inp["K"], inp["V"], sel_tok[:, None, :], 690)

@@ -17,7 +17,7 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import GpuRun, oracle_scores, to_f64, check_selection
+from samkv_testlib import DeviceRun, oracle_scores, to_f64, check_selection
 
 pytestmark = pytest.mark.gpu
 
@@ -29,7 +29,7 @@ def ulp(x, dtype):
 
 def block_run(w):
     inp = synth.make_inputs(w, "cuda")
-    run = GpuRun(w, inp)
+    run = DeviceRun(w, inp)
     Kbar = torch.full((w.n_layers, w.batch, w.n_kv_heads, run.U_tot, w.head_dim), 7.0, dtype=w.torch_dtype, device="cuda")
     B.samkv_block_means(run.handle, run.shape, inp["K"], Kbar)
     scores = torch.full_like(run.scores, -5.0)

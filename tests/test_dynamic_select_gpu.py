@@ -18,14 +18,14 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import GpuRun
+from samkv_testlib import DeviceRun
 
 pytestmark = pytest.mark.gpu
 
 
 def gpu_scores(w, scores=None):
     inp = synth.make_inputs(w, "cuda")
-    run = GpuRun(w, inp)
+    run = DeviceRun(w, inp)
     if scores is None:
         B.samkv_score(run.handle, run.shape, inp["K"], inp["Q"], w.q_tokens, inp["Qloc"], inp["Qloc"].shape[3], 1,
                       run.scores, run.qhat)

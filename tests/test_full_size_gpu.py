@@ -8,7 +8,7 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import (GpuRun, check_attention, check_compact, check_scores, check_selection, check_update,
+from samkv_testlib import (DeviceRun, check_attention, check_compact, check_scores, check_selection, check_update,
                            oracle_scores, to_f64)
 
 pytestmark = pytest.mark.gpu
@@ -26,7 +26,7 @@ def test_cfg2_full_size_sampled_slabs():
     fusion update of 15 % of the kept tokens, attention with the appended 64-token chunk."""
     w = synth.CONFIGS["cfg2"]
     inp = synth.make_inputs(w, DEV)
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     assert run.S == 4600 and run.poll() == 0
     samples = [(0, 0), (17, 2), (31, 3)]
@@ -77,7 +77,7 @@ def test_cfg3_full_size_decode_128_steps():
     steps of one token each appending to the compact cache; sampled batch elements follow every step."""
     w = synth.CONFIGS["cfg3"]
     inp = synth.make_inputs(w, DEV)
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     assert run.S == 3070
     sample_b = [0, 13, 31]
@@ -125,7 +125,7 @@ def test_cfg4_stress_budget_sweep(budget_bp):
     must equal full attention over the concatenated contexts (oracle run on the original K/V)."""
     w = synth.CONFIGS["cfg4"].replace(budget_bp=budget_bp)
     inp = synth.make_inputs(w, DEV)
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     assert run.S == {500: 5100, 1500: 15350, 3000: 30700, 10000: 102400}[budget_bp]
     sel = run.sel[0, 0].cpu().numpy()

@@ -11,7 +11,7 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import (GpuRun, check_attention, check_compact, check_scores, check_selection, check_update,
+from samkv_testlib import (DeviceRun, check_attention, check_compact, check_scores, check_selection, check_update,
                            oracle_k_units, oracle_scores, to_f64)
 
 pytestmark = pytest.mark.gpu
@@ -21,7 +21,7 @@ DEV = "cuda:0"
 def full_check(w, inp=None, k_units=None, use_bias=True, with_qloc=True, append=True, layers=None, batches=None):
     """Sparsify + prefill attention for a workload; every stage against the oracle."""
     inp = inp if inp is not None else {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp, k_units=k_units, use_bias=use_bias, with_qloc=with_qloc).sparsify()
+    run = DeviceRun(w, inp, k_units=k_units, use_bias=use_bias, with_qloc=with_qloc).sparsify()
     if k_units is None:
         assert run.k_units == oracle_k_units(w)
     torch.cuda.synchronize()
@@ -138,7 +138,7 @@ def test_update_overwrite_and_fusion(mode, dtype):
     w = synth.CONFIGS["cfg2"].replace(name="cfg2_small", n_layers=2, batch=2, ctx_lens=(384, 256, 512), dtype=dtype,
                                       q_tokens=16)
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     sel = run.sel.cpu().numpy()
     toks0 = np.stack([[O.units_to_tokens(sel[l, b, 0], w.ctx_offsets, 1) for b in range(w.batch)]
                       for l in range(w.n_layers)])
@@ -167,7 +167,7 @@ def test_decode_steps_append_to_compact_cache():
     """Reduced cfg3: sparsify, prefill a 32-token chunk, then decode steps of one token each."""
     w = synth.CONFIGS["cfg3"].replace(name="cfg3_small", batch=3, ctx_lens=(512, 768, 300), decode_steps=12)
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
     Kc_ref = [to_f64(run.Kc[0, b]) for b in range(w.batch)]
     Vc_ref = [to_f64(run.Vc[0, b]) for b in range(w.batch)]
@@ -202,7 +202,7 @@ def test_results_are_deterministic():
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
     outs = []
     for _ in range(3):
-        run = GpuRun(w, inp).sparsify()
+        run = DeviceRun(w, inp).sparsify()
         Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
         outs.append((run.scores.clone(), run.sel.clone(), run.Kc.clone(), Og.clone(), lse.clone()))
     for o in outs[1:]:
@@ -213,7 +213,7 @@ def test_results_are_deterministic():
 def test_error_codes_launch_nothing():
     w = synth.CONFIGS["cfg0"]
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     sel_before = run.sel.clone()
     with pytest.raises(B.SamkvError) as e:
@@ -245,7 +245,7 @@ def test_append_past_capacity_is_reported_not_fatal():
     """A full cache: the append is skipped, a device check is recorded, the context stays usable."""
     w = synth.CONFIGS["cfg0"]
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp, extra_capacity=8).sparsify()               # room for 8 tokens, chunk has 16
+    run = DeviceRun(w, inp, extra_capacity=8).sparsify()               # room for 8 tokens, chunk has 16
     Og, _ = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
     assert run.poll() == 7
     assert int(run.cache_len[0, 0]) == run.S
@@ -259,7 +259,7 @@ def test_compact_gathers_v_rows_from_pinned_host_memory():
     """V may stay in pinned host memory; only the kept rows cross the bus.  Same bits as with V on the device."""
     w = synth.CONFIGS["cfg1"]
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp).sparsify()
+    run = DeviceRun(w, inp).sparsify()
     torch.cuda.synchronize()
     Kc_dev, Vc_dev = run.Kc.clone(), run.Vc.clone()
     V_host = inp["V"].cpu().pin_memory()
@@ -334,7 +334,7 @@ def test_chunked_prefill_on_the_tensor_memory_kernel():
     length and the rows the previous call left, then a cache-only call must see all three chunks."""
     w = synth.CONFIGS["cfg1"].replace(name="cfg1_chunks", batch=2, q_tokens=64, ctx_lens=(1024, 700, 1300))
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
-    run = GpuRun(w, inp, extra_capacity=3 * 64).sparsify()
+    run = DeviceRun(w, inp, extra_capacity=3 * 64).sparsify()
     torch.cuda.synchronize()
     Kc_ref = [to_f64(run.Kc[0, b]) for b in range(w.batch)]
     Vc_ref = [to_f64(run.Vc[0, b]) for b in range(w.batch)]

@@ -9,7 +9,7 @@ import torch
 from oracle import samkv_oracle as O
 from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
-from samkv_testlib import GpuRun, check_attention
+from samkv_testlib import DeviceRun, check_attention
 
 pytestmark = pytest.mark.gpu
 
@@ -18,7 +18,7 @@ def protected_run(w):
     inp = synth.make_inputs(w, "cuda")
     shape = B.Shape.from_workload(w)
     prot, _, _ = B.samkv_layout(shape)
-    run = GpuRun(w, inp, k_units=prot)
+    run = DeviceRun(w, inp, k_units=prot)
     return run, inp, prot
 
 
@@ -79,7 +79,7 @@ def test_no_selection_ablation_is_a_subset_of_the_selected_cache():
     """Every row of the protected-only cache also sits in the cache built with a budget, in the same order."""
     w = synth.CONFIGS["cfg1"]
     inp = synth.make_inputs(w, "cuda")
-    full = GpuRun(w, inp).sparsify()
+    full = DeviceRun(w, inp).sparsify()
     run, _, prot = protected_run(w)
     Kc, Vc, cache_len, inv = compact_protected(run, inp)
     torch.cuda.synchronize()
