@@ -485,7 +485,7 @@ def job_throughput(w, world: int, ms_per_step: float) -> float:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="samkv", choices=["samkv", "reference"])
     ap.add_argument("--workload", default="cfg2")
