@@ -299,6 +299,57 @@ class Pipeline:
         return n + self.w.n_layers * self.w.decode_steps * KERNELS_PER_CALL["attn_append_split"]
 
 
+def widened_rows_ms(pipe: Pipeline, reps: int = 5):
+    """Device time of the calls beyond the fixed-budget path, on the workload's own tensors, outside the timed
+    region: dynamic selection (Top-P, cross-context Top-K, gather of its unit lists), cross-layer alignment,
+    protected-only gather.  Block representatives are timed only when the workload scores blocks (block_size > 1)."""
+    w, B = pipe.w, pipe.B
+    dev = pipe.dev
+    L, Bt, Hkv, D = w.n_layers, w.batch, w.n_kv_heads, w.n_ctx
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    out = {}
+    P = torch.zeros((Bt, D), dtype=torch.float32, device=dev)
+    star = list(range(max(0, L - 4), L))
+    out["topp"] = timed(lambda: B.samkv_topp(pipe.handle, pipe.shape, pipe.scores, star, None, None, P))
+    P_row = [min(1.0, max(0.0, float(x))) for x in P[0].cpu()]
+    cand, K, S_u, S = B.samkv_topp_plan(pipe.shape, P_row)
+    sel = torch.empty((L, Bt, Hkv, S_u), dtype=torch.int32, device=dev)
+    scratch = torch.empty(B.samkv_select_cross_scratch_bytes(pipe.shape, cand), dtype=torch.uint8, device=dev)
+    out["select_cross"] = timed(lambda: B.samkv_select_cross(pipe.handle, pipe.shape, pipe.scores, cand, scratch, sel))
+    if S <= pipe.capacity:
+        out["compact_units"] = timed(lambda: B.samkv_compact_units(pipe.handle, pipe.shape, pipe.inp["K"], pipe.inp["V"], sel,
+                                                                  S_u, pipe.Kc, pipe.Vc, pipe.capacity, pipe.cache_len,
+                                                                  pipe.inv_map))
+    out["dynamic_kept_tokens"] = S
+    out["compact_protected"] = timed(lambda: B.samkv_compact_protected(pipe.handle, pipe.shape, pipe.inp["K"], pipe.inp["V"],
+                                                                      pipe.Kc, pipe.Vc, pipe.capacity, pipe.cache_len,
+                                                                      pipe.inv_map))
+    pipe.sparsify()                                        # restore the fixed-budget cache and its inverse map
+    if pipe.R > 0:
+        flags = torch.empty((L, Bt, w.l_tot), dtype=torch.uint8, device=dev)
+        merged = torch.empty((Bt, w.l_tot), dtype=torch.int32, device=dev)
+        merged_len = torch.empty((Bt,), dtype=torch.int32, device=dev)
+        run_ids = torch.empty((L, Bt, min(w.l_tot, L * pipe.R)), dtype=torch.int32, device=dev)
+        run_len = torch.empty((L, Bt), dtype=torch.int32, device=dev)
+        out["align"] = timed(lambda: B.samkv_align(pipe.handle, pipe.shape, pipe.inv_map, pipe.tok_ids, flags, merged,
+                                                   merged_len, run_ids, run_len))
+    torch.cuda.synchronize()
+    if B.samkv_poll_status(pipe.handle) != 0:
+        raise RuntimeError("device-side check failed in the widened rows")
+    return out
+
+
 def e2e_steps(pipe: Pipeline, steps: int, warmup: int):
     """Same step, but every step's inputs start in pinned HOST memory and the result is read back.
     Per layer, a copy stream brings that layer's K and query rows over while the compute stream works on
@@ -577,6 +628,7 @@ def main():
             phase_ms[n1] = phase_ms.get(n1, 0.0) + a.elapsed_time(b) / n_seq
     sequential_ms = sum(phase_ms.values())
     phase_ms["score"] = timed_phase_ms["score"]          # the roofline figure comes from the timed steps
+    widened = widened_rows_ms(pipe) if (rank == 0 and w.decode_steps == 0 and not profiling_case) else None
 
     ms_per_step = elapsed_ms / args.steps
     value = job_throughput(w, world, ms_per_step)
@@ -601,7 +653,7 @@ def main():
                      "schedule": ("score+select, then %d layer groups: gather+update overlapped with attention on a second stream"
                                   % pipe.groups) if pipe.groups > 1 else "in order on one stream",
                      "timed_phase_ms": timed_phase_ms, "in_order_ms_per_step": sequential_ms,
-                     "phase_ms": phase_ms,
+                     "phase_ms": phase_ms, "other_calls_ms": widened,
                      "phase_gbs": {k: ab[k] / (phase_ms[k] / 1e3) / 1e9 for k in ("score", "compact", "update", "attn", "decode") if phase_ms.get(k, 0) > 0}},
         "roofline": {"kernel": "score_stream_kernel (with the pooled-query kernel that precedes it in samkv_score)", "bound": "hbm",
                      "achieved": score_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
