@@ -363,3 +363,17 @@ def test_chunked_prefill_on_the_tensor_memory_kernel():
         assert np.abs(to_f64(O_last[b]) - out).max() <= 2e-2
         assert np.abs(to_f64(lse_last[b]) - l2).max() <= 2e-2
         assert np.array_equal(to_f64(run.Kc[0, b])[:, :n], Kc_ref[b][:, :n])
+
+
+@pytest.mark.parametrize("ctx_lens,T_q,Hq,Hkv,budget_bp", [
+    ((40, 30), 32, 8, 2, 10000),          # 128 rows, one partial KV tile: cache (70) + chunk (32) < 128 slots
+    ((100, 90), 129, 2, 2, 10000),        # G = 1, 129 rows: a second query tile with a single real row
+    ((200, 56), 16, 32, 2, 10000),        # G = 16, 256 rows; the chunk crosses the 256-slot tile boundary
+    ((700, 900, 333), 50, 12, 2, 3000),   # G = 6 (rows of one token straddle lane quarters), 300 rows, ragged
+    ((2048,) * 3, 128, 16, 2, 10000),     # 1024 rows per KV head: eight query tiles share each K/V tile
+])
+def test_tensor_memory_attention_edge_shapes(ctx_lens, T_q, Hq, Hkv, budget_bp):
+    """Shapes that exercise the tcgen05 kernels' corners: partial tiles, single-row query tiles, large groups."""
+    w = synth.ragged_workload(ctx_lens=ctx_lens, dtype="bf16", head_dim=128, n_q_heads=Hq, n_kv_heads=Hkv,
+                              q_tokens=T_q, n_init=4, n_local=8, budget_bp=budget_bp, seed=1234 + T_q)
+    full_check(w)
