@@ -307,3 +307,20 @@ def test_dynamic_end_to_end_attention():
     assert int(run.cache_len[0, 0]) == S + w.q_tokens
     check_attention(w, torch.from_numpy(Kc_or), torch.from_numpy(Vc_or), S, inp["Qa"][0, 0], inp["Kq"][0, 0],
                     inp["Vq"][0, 0], Og[0], lse[0])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_dynamic_random_shapes(seed):
+    """Seeded random small workloads through Top-P, cross-context Top-K and the gather of its unit lists."""
+    r = np.random.default_rng(7000 + seed)
+    Bsz = int(2 ** r.integers(0, 5))
+    n_ctx = int(r.integers(1, 7))
+    lens = tuple(int(x) for x in r.integers(3 * Bsz + 1, 40 * Bsz + 300, size=n_ctx))
+    Hkv = int(r.choice([1, 2, 4]))
+    w = synth.ragged_workload(name=f"dynfuzz{seed}", ctx_lens=lens, dtype=str(r.choice(["bf16", "f32"])),
+                              head_dim=int(r.choice([64, 128])), n_q_heads=2 * Hkv, n_kv_heads=Hkv,
+                              q_tokens=int(r.integers(1, 20)), block_size=Bsz, n_init=Bsz * int(r.integers(0, 3)),
+                              n_local=Bsz * int(r.integers(1, 4)), seed=7000 + seed)
+    w = dataclasses.replace(w, n_layers=int(r.integers(1, 4)), batch=int(r.integers(1, 3)))
+    P_override = None if seed % 2 == 0 else [float(x) for x in r.random(n_ctx)]
+    run_dynamic(w, star=list(range(w.n_layers))[-2:], P_override=P_override)

@@ -377,3 +377,24 @@ def test_tensor_memory_attention_edge_shapes(ctx_lens, T_q, Hq, Hkv, budget_bp):
     w = synth.ragged_workload(ctx_lens=ctx_lens, dtype="bf16", head_dim=128, n_q_heads=Hq, n_kv_heads=Hkv,
                               q_tokens=T_q, n_init=4, n_local=8, budget_bp=budget_bp, seed=1234 + T_q)
     full_check(w)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_against_the_oracle(seed):
+    """Seeded random small workloads: every stage of the path against the oracle (shapes no hand-written case covers)."""
+    r = np.random.default_rng(9000 + seed)
+    Bsz = int(2 ** r.integers(0, 5))                                   # block size 1 .. 16
+    n_ctx = int(r.integers(1, 7))
+    lens = tuple(int(x) for x in r.integers(3 * Bsz + 1, 40 * Bsz + 200, size=n_ctx))
+    G = int(r.choice([1, 2, 4, 8]))
+    Hkv = int(r.choice([1, 2, 4]))
+    dtype = str(r.choice(["bf16", "f32"]))
+    d = int(r.choice([64, 128]))
+    T_q = int(r.integers(1, 70))
+    n_init = Bsz * int(r.integers(0, 3))
+    n_local = Bsz * int(r.integers(1, 4))
+    w = synth.ragged_workload(name=f"fuzz{seed}", ctx_lens=lens, dtype=dtype, head_dim=d, n_q_heads=G * Hkv,
+                              n_kv_heads=Hkv, q_tokens=T_q, block_size=Bsz, n_init=n_init, n_local=n_local,
+                              budget_bp=int(r.integers(500, 10001)), seed=9000 + seed)
+    w = w.replace(n_layers=int(r.integers(1, 3)), batch=int(r.integers(1, 3)))
+    full_check(w)
