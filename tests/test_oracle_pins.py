@@ -587,22 +587,36 @@ def test_cross_context_select_properties():
 # Section 3.3: blank-block alignment and the two recomputation rules
 # ------------------------------------------------------------------------------------------
 def test_align_layers_the_four_cases_of_the_recomputation_figure():
-    """Two layers, one head.  Tokens: 0 lower layer recomputed / upper not; 1 neither; 2 upper recomputed /
-    lower not, and blank in the lower layer; 3 both; 4 blank everywhere but listed; 5 upper recomputed, lower
-    kept and not recomputed.  Expected flags follow the paper's discussion of its examples 1-4."""
-    K, R, Out, Pad = O.FLAG_KEPT, O.FLAG_RECOMPUTE, O.FLAG_OUTPUT, O.FLAG_PAD_REUSE
-    inv = np.full((2, 1, 6), -1, dtype=np.int32)
-    inv[0, 0, [0, 1, 3, 5]] = [0, 1, 2, 3]          # lower layer keeps 0, 1, 3, 5 (2 and 4 are blanks)
-    inv[1, 0, [0, 1, 2, 3, 5]] = [0, 1, 2, 3, 4]    # upper layer keeps 0, 1, 2, 3, 5
-    tok = np.array([[0, 3, 4, -1], [2, 3, 5, -1]])
+    """tests/golden/recompute_figure_cases.txt: the four token cases of the paper's recomputation figure (plus two
+    corner tokens) as a two-layer, one-head example with the flags the text prescribes for each."""
+    letters = {"K": O.FLAG_KEPT, "R": O.FLAG_RECOMPUTE, "O": O.FLAG_OUTPUT, "P": O.FLAG_PAD_REUSE}
+    rows = []
+    with open(os.path.join(GOLDEN, "recompute_figure_cases.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            body = line.split("=")[1]
+            bits, lower, upper = [x.strip() for x in body.split("|")]
+            rows.append(([int(x) for x in bits.split(",")], lower, upper))
+    T = len(rows)
+    assert T == 6
+    inv = np.full((2, 1, T), -1, dtype=np.int32)
+    lists = [[], []]
+    for t, (bits, _, _) in enumerate(rows):
+        for n in range(2):
+            if bits[n]:
+                inv[n, 0, t] = int((inv[n, 0, :t] >= 0).sum())          # slots in token order
+            if bits[2 + n]:
+                lists[n].append(t)
+    R = max(len(x) for x in lists) + 1
+    tok = np.array([x + [-1] * (R - len(x)) for x in lists])
     flags, merged, run = O.align_layers(inv, tok)
-    assert flags[:, 0].tolist() == [K | R, K]                 # (1) K/V refreshed below, no output needed
-    assert flags[:, 1].tolist() == [K, K]                     # (2) nothing to do
-    assert flags[:, 2].tolist() == [Out | Pad, K | R]         # (3) output below from the prefilled entry
-    assert flags[:, 3].tolist() == [K | R | Out, K | R]       # (4)
-    assert flags[:, 4].tolist() == [0, 0]                     # listed but blank: nothing to refresh
-    assert flags[:, 5].tolist() == [K | Out, K | R]           # output below, K/V reused from the compact cache
-    assert merged.tolist() == [0, 1, 2, 3, 5]
+    for t, (_, lower, upper) in enumerate(rows):
+        for n, want in enumerate((lower, upper)):
+            expect = sum(letters[ch] for ch in want if ch in letters)
+            assert flags[n, t] == expect, f"token {t + 1} layer {n}: {flags[n, t]} != {want}"
+    assert merged.tolist() == [0, 1, 2, 3, 5]                              # token 5 is kept by no layer
     assert run[0].tolist() == [0, 2, 3, 5] and run[1].tolist() == [2, 3, 5]
 
 
