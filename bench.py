@@ -41,7 +41,7 @@ HBM_FALLBACK_GBS = 6650.0
 # profiles/score_stream_kernel_cfg2_2layers.md (dram read + write of one launch / rows of that launch);
 # traffic grows in proportion to the rows (no reuse), so a full launch is rows x this figure.
 SCORE_KERNEL_DRAM_BYTES_PER_ROW = 260.0
-KERNELS_PER_CALL = {"score": 2, "select": 1, "compact": 1, "update": 1, "attn_append_split": 3}
+KERNELS_PER_CALL = {"score": 2, "select": 1, "compact": 1, "update": 1}      # samkv_attn: asked from the library
 
 
 def measured_peaks():
@@ -295,8 +295,10 @@ class Pipeline:
             per_group += KERNELS_PER_CALL["update"]
         # the timed schedule gathers and updates group by group
         n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + self.groups * per_group
-        n += self.w.n_layers * KERNELS_PER_CALL["attn_append_split"]
-        return n + self.w.n_layers * self.w.decode_steps * KERNELS_PER_CALL["attn_append_split"]
+        B = self.B
+        n += self.w.n_layers * B.samkv_attn_kernel_count(self.handle_attn, self.shape1, self.w.q_tokens, self.capacity, True)
+        return n + self.w.n_layers * self.w.decode_steps * B.samkv_attn_kernel_count(self.handle, self.shape, 1,
+                                                                                    self.capacity, True)
 
 
 def widened_rows_ms(pipe: Pipeline, reps: int = 5):

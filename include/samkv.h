@@ -239,6 +239,12 @@ samkv_status_t samkv_compact_units(samkv_handle_t h, const samkv_shape_t* shape,
                                    const int32_t* sel, int32_t S_u, void* Kc, void* Vc, int32_t cache_capacity,
                                    int32_t* cache_len, int32_t* inv_map, void* stream);
 
+/* Number of kernels one samkv_attn call with these sizes launches on the device of `h` (append of the chunk when
+ * `appended`, the attention kernel, the merge of KV splits where the attention kernel does not merge them itself).
+ * For launch accounting; returns 0 for arguments samkv_attn would refuse. */
+int32_t samkv_attn_kernel_count(samkv_handle_t h, const samkv_shape_t* shape, int32_t T_q, int32_t cache_capacity,
+                                int32_t appended);
+
 /* ---- block representatives (Sec. 3.2: "each block is represented by the mean vector of its token caches") --- */
 
 /* Kbar[l,b,h,u,:] = mean over the tokens of unit u of K[l,b,h,t,:] (fp32 sum in a fixed order, one rounding to the

@@ -356,6 +356,18 @@ samkv_status_t samkv_attn(samkv_handle_t handle, const samkv_shape_t* shape, int
                                h->workspace + ws_off, plan, h->d_status, static_cast<cudaStream_t>(stream)));
 }
 
+int32_t samkv_attn_kernel_count(samkv_handle_t handle, const samkv_shape_t* shape, int32_t T_q, int32_t cache_capacity,
+                                int32_t appended) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  Layout lo;
+  if (h == nullptr || make_layout(shape, &lo) != SAMKV_OK || T_q < 1 || cache_capacity < 1) return 0;
+  const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count);
+  const bool self_merge = shape->dtype == SAMKV_BF16 && attn_tc3_merges_in_cluster(plan);
+  int n = 1 + (appended ? 1 : 0);
+  if ((plan.n_splits > 1 || appended) && !self_merge) ++n;
+  return n;
+}
+
 samkv_status_t samkv_topp(samkv_handle_t handle, const samkv_shape_t* shape, const float* scores,
                           const int32_t* star_layers, int32_t n_star, const int32_t* max_units,
                           const int32_t* min_units, float* P_out, void* stream) {

@@ -23,10 +23,9 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
                             cudaStream_t stream);
-cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
-                            const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
-                            float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
-                            cudaStream_t stream);
+cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
+                            const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
+                            float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Plan: how many packed rows a CTA takes and into how many KV splits a (batch, kv head) is cut.
@@ -344,7 +343,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
         Kl, Vl, len_l, (const T*)Q, (T*)O, lse, part_o, part_ml, Hq, Hkv, T_q, capacity, appended, scale,
         plan.n_splits, row_tiles);
   }
-  if (plan.n_splits > 1 || appended) {
+  if ((plan.n_splits > 1 || appended) && !(sizeof(T) == 2 && attn_tc3_merges_in_cluster(plan))) {
     const long long blocks = plan.n_splits > 1 ? (long long)((out_rows + 3) / 4) : 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);

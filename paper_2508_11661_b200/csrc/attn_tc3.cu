@@ -15,6 +15,9 @@
 //               P ready -> O += P V -> next S.
 //   warp  9     loader: K (3 stages) and V (2 stages) tiles arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle)
 // Tensor memory: S buffers [0,128) and [128,256), O [256,384).
+// With exactly two KV splits the grid is launched in clusters of two CTAs (the two splits of one query tile): the
+// second hands its (m, l, O) to the first through distributed shared memory between two cluster barriers, and the
+// first writes the final rows; every thread of both CTAs walks through both barriers on every path.
 // All hand-offs are mbarriers polled by one lane per warp; every wait is bounded and a timeout is recorded as a
 // device check, after which the CTA drains and frees its tensor memory.  The TMA loads read this GPU's memory only
 // and use no multicast.
@@ -52,19 +55,28 @@ enum Bar {
 
 }  // namespace tc3
 
+// kPair: the grid is launched in clusters of two CTAs, the two KV splits of one (batch, kv head, query tile).  The
+// CTA of the second split hands its (m, l, O) to the first one through distributed shared memory, which writes the
+// final rows: no partial results in global memory and no merge kernel.  The cache length of an appended chunk is then
+// bumped by the last CTA of the grid to finish (a counter in the workspace's status block).
+template <bool kPair>
 __global__ void __launch_bounds__(tc3::kThreads, 1)
 attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                const int32_t* __restrict__ cache_len, const __nv_bfloat16* __restrict__ Q,
+                int32_t* cache_len, const __nv_bfloat16* __restrict__ Q,
                 __nv_bfloat16* __restrict__ O, float* __restrict__ lse, float* __restrict__ part_o,
                 float2* __restrict__ part_ml, int Hq, int Hkv, int T_q, int capacity, int appended, float scale,
                 int n_splits, int row_tiles, int* __restrict__ d_status) {
   using namespace tc3;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
-  if ((base & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicMax(d_status, (int)CHECK_SMEM_ALIGNMENT);
-    return;
-  }
+  // A misaligned buffer (never seen: the declaration asks for 1024 bytes) is reported and the CTA does no tile work,
+  // but it still walks through every barrier below, so its cluster partner is not left waiting.
+  const bool bad_smem = (base & 1023u) != 0;
+  if (bad_smem && threadIdx.x == 0) atomicMax(d_status, (int)CHECK_SMEM_ALIGNMENT);
+  auto pair_sync = [&]() {                                    // all threads of both CTAs of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  };
   const uint32_t sQ = base + kOffQ, sK = base + kOffK, sV = base + kOffV, sBar = base + kOffBar;
   float* x_max = reinterpret_cast<float*>(smem_raw + kOffX);          // [parity][half][row]
   float* x_sum = x_max + 2 * kParts * kBM;                            // [part][row]
@@ -133,7 +145,7 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const int tps = (n_tiles + n_splits - 1) / n_splits;
   const int tile0 = split * tps;
   const int tile1 = min(min(tile0 + tps, n_tiles), (cta_visible + kBN - 1) / kBN);
-  const int nt = max(tile1 - tile0, 0);
+  const int nt = bad_smem ? 0 : max(tile1 - tile0, 0);
 
   if (warp < kSoftmaxWarps) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -188,6 +200,7 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       load_v(j);
       if (j + 2 < nt) load_k(j + 2);
     }
+    if constexpr (kPair) { pair_sync(); pair_sync(); }
   } else if (warp == kMmaWarp) {
     // ================= MMA issuer =================
     if (lane == 0 && nt > 0) {
@@ -235,6 +248,8 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       }
       mma_commit(bar(O_FINAL));
     }
+    __syncwarp();
+    if constexpr (kPair) { pair_sync(); pair_sync(); }
   } else {
     // ================= softmax warps =================
     const int wl = warp & 3;                                    // tensor-memory lane quarter
@@ -331,6 +346,81 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     float l_row = 0.f;
 #pragma unroll
     for (int pp = 0; pp < kParts; ++pp) l_row += x_sum[pp * kBM + row_in_tile];
+    if constexpr (kPair) {
+      // ---- merge of the two KV splits inside the cluster ----
+      // Exchange area in the first CTA's K ring: O parts [part][row][kPartCols] fp32 with the 16-byte chunks of a row
+      // XOR-swizzled by the row (threads of a warp write different rows), then (m, l) per row.
+      const uint32_t xo_local = sK + (uint32_t)((part * kBM + row_in_tile) * kPartCols * 4);
+      const uint32_t xml_local = sK + (uint32_t)(kParts * kBM * kPartCols * 4 + row_in_tile * 8);
+      constexpr int kChunks = kPartCols / 4;                    // 16-byte chunks per part of a row
+      pair_sync();                                              // both CTAs are past their last MMA: the rings are free
+      if (split == 1) {
+        uint32_t xo_remote, xml_remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(xo_remote) : "r"(xo_local));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(xml_remote) : "r"(xml_local));
+#pragma unroll 1
+        for (int c0 = 0; c0 < kPartCols; c0 += 32) {
+          float o[32];
+          if (nt > 0) {
+            tmem_ld32(tO + c0, o);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = 0.f;
+          }
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const int chunk = ((c0 + i) >> 2) ^ (row_in_tile & (kChunks - 1));
+            asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(xo_remote + chunk * 16), "f"(o[i]),
+                         "f"(o[i + 1]), "f"(o[i + 2]), "f"(o[i + 3]) : "memory");
+          }
+        }
+        if (part == 0)
+          asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(xml_remote), "f"(m), "f"(l_row) : "memory");
+      }
+      pair_sync();                                              // the second split's numbers have landed
+      if (split == 0) {
+        float m1, l1;
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(m1), "=f"(l1) : "r"(xml_local) : "memory");
+        const bool has0 = l_row > 0.f, has1 = l1 > 0.f;
+        const float M = fmaxf(has0 ? m : -INFINITY, has1 ? m1 : -INFINITY);
+        const float w0 = has0 ? fast_exp2(m - M) : 0.f, w1 = has1 ? fast_exp2(m1 - M) : 0.f;
+        const float L = l_row * w0 + l1 * w1;
+        const float inv = L > 0.f ? 1.0f / L : 0.f;
+        const float a0 = w0 * inv, a1 = w1 * inv;
+        const bool store = my_row < rows_total && *s_fail == 0;
+        const int rr = min(my_row, rows_total - 1);
+        const int t = rr / G, hq = h * G + rr % G;
+        const size_t orow = ((size_t)b * T_q + t) * Hq + hq;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kPartCols; c0 += 32) {
+          float o[32];
+          if (nt > 0) {
+            tmem_ld32(tO + c0, o);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = 0.f;
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const int chunk = ((c0 + i) >> 2) ^ (row_in_tile & (kChunks - 1));
+            float4 o1;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o1.x), "=f"(o1.y), "=f"(o1.z), "=f"(o1.w)
+                         : "r"(xo_local + chunk * 16) : "memory");
+            pk[i >> 1] = pack_bf16(fmaf(o[i], a0, o1.x * a1), fmaf(o[i + 1], a0, o1.y * a1));
+            pk[(i >> 1) + 1] = pack_bf16(fmaf(o[i + 2], a0, o1.z * a1), fmaf(o[i + 3], a0, o1.w * a1));
+          }
+          if (store) {
+            __nv_bfloat16* op = O + orow * kD + part * kPartCols + c0;
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+              *reinterpret_cast<uint4*>(op + i * 2) = make_uint4(pk[i], pk[i + 1], pk[i + 2], pk[i + 3]);
+          }
+        }
+        if (store && part == 0 && lse != nullptr)
+          lse[((size_t)b * Hq + hq) * T_q + t] = L > 0.f ? M * kLn2 + logf(L) : -INFINITY;
+      }
+    } else {
     // ---- write this thread's part of the row ----
     const bool failed = *s_fail != 0;
     const bool store = my_row < rows_total && !failed;
@@ -373,6 +463,7 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         part_ml[orow * n_splits + split] = make_float2(l_row > 0.f ? m * kLn2 : -INFINITY, l_row);
       }
     }
+    }  // !kPair
   }
 
   // ---- teardown: every role arrives here, then the allocating warp frees tensor memory ----
@@ -380,16 +471,30 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   __syncthreads();
   pdl_launch_dependents();      // results are written: the merge kernel may be scheduled (it still waits for our exit)
   if (tid == 0 && *s_fail) atomicMax(d_status, (int)CHECK_WAIT_TIMEOUT);
+  if constexpr (kPair) {
+    // no merge kernel follows: the last CTA of the grid to get here knows that every CTA has read cache_len
+    if (tid == 0 && appended) {
+      int* ticket = d_status + kAttnTicketInt;
+      __threadfence();
+      if (atomicAdd(ticket, 1) == (int)gridDim.x - 1) {
+        const int Bt = (int)(gridDim.x / (unsigned)(n_splits * row_tiles * Hkv));
+        for (int bb = 0; bb < Bt; ++bb) {
+          const int cur = cache_len[bb];
+          if (cur >= 0 && cur + T_q <= capacity) cache_len[bb] = cur + T_q;
+        }
+        *ticket = 0;
+      }
+    }
+  }
   if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
 
-cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity,
-                            const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
-                            float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
-                            cudaStream_t stream) {
+cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
+                            const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
+                            float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream) {
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = T_q * G;
   const int row_tiles = (rows + tc3::kBM - 1) / tc3::kBM;
@@ -399,7 +504,9 @@ cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* 
   if (!tc::make_kv_map(&tmK, Kc, capacity, s.batch * s.n_kv_heads) ||
       !tc::make_kv_map(&tmV, Vc, capacity, s.batch * s.n_kv_heads))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_tc3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc3::kSmemBytes);
+  const bool pair = attn_tc3_merges_in_cluster(plan);
+  auto kern = pair ? attn_tc3_kernel<true> : attn_tc3_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc3::kSmemBytes);
   if (e != cudaSuccess) return e;
   // Launched so that it may start while the kernel before it in the stream (the append of the chunk) is still
   // running: set-up and the Q loads need nothing from it; one wait precedes everything that does.
@@ -408,14 +515,18 @@ cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* 
   cfg.blockDim = dim3(tc3::kThreads);
   cfg.dynamicSmemBytes = tc3::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, attn_tc3_kernel, tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (__nv_bfloat16*)O, lse,
-                            part_o, part_ml, s.n_q_heads, s.n_kv_heads, T_q, capacity, appended, scale, plan.n_splits,
-                            row_tiles, d_status);
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[0].val.programmaticStreamSerializationAllowed = 1;
+  attrs[1].id = cudaLaunchAttributeClusterDimension;
+  attrs[1].val.clusterDim.x = 2;
+  attrs[1].val.clusterDim.y = 1;
+  attrs[1].val.clusterDim.z = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = pair ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kern, tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (__nv_bfloat16*)O, lse, part_o,
+                            part_ml, s.n_q_heads, s.n_kv_heads, T_q, capacity, appended, scale, plan.n_splits, row_tiles,
+                            d_status);
 }
 
 }  // namespace samkv

@@ -73,6 +73,11 @@ struct AttnPlan {
   size_t partial_bytes;
 };
 AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count);
+// The 128-row tcgen05 kernel with exactly two KV splits merges them inside a two-CTA cluster: no merge kernel.
+inline bool attn_tc3_merges_in_cluster(const AttnPlan& p) { return p.rows_per_cta == 128 && p.n_splits == 2; }
+// Status block of the workspace (256 bytes, zero between calls): int 0 is the device check word, this int counts the
+// finished CTAs of an attention grid that bumps cache_len itself.
+constexpr int kAttnTicketInt = 32;
 cudaError_t launch_attn(const samkv_shape_t& s, int layer, void* Kc, void* Vc, int capacity, int32_t* cache_len,
                         const void* Q, int T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
                         void* partial_ws, const AttnPlan& plan, int* d_status, cudaStream_t stream);
