@@ -16,8 +16,8 @@
 //   warp  9     loader: K (3 stages) and V (2 stages) tiles arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle)
 // Tensor memory: S buffers [0,128) and [128,256), O [256,384).
 // With exactly two KV splits the grid is launched in clusters of two CTAs (the two splits of one query tile): the
-// second hands its (m, l, O) to the first through distributed shared memory between two cluster barriers, and the
-// first writes the final rows; every thread of both CTAs walks through both barriers on every path.
+// CTAs swap the (m, l, O) of half of the rows each through distributed shared memory between two cluster barriers and
+// each writes the final result of its half; every thread of both CTAs walks through both barriers on every path.
 // All hand-offs are mbarriers polled by one lane per warp; every wait is bounded and a timeout is recorded as a
 // device check, after which the CTA drains and frees its tensor memory.  The TMA loads read this GPU's memory only
 // and use no multicast.
@@ -354,10 +354,14 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const uint32_t xml_local = sK + (uint32_t)(kParts * kBM * kPartCols * 4 + row_in_tile * 8);
       constexpr int kChunks = kPartCols / 4;                    // 16-byte chunks per part of a row
       pair_sync();                                              // both CTAs are past their last MMA: the rings are free
-      if (split == 1) {
+      // Each CTA merges half of the rows: rows [0,64) end up in the CTA of the first split, rows [64,128) in the
+      // other one, so both CTAs send 32 KB, merge 64 rows and write 16 KB instead of one of them doing it all.
+      const bool mine = (row_in_tile < kBM / 2) == (split == 0);          // this CTA writes this row's result
+      if (!mine) {
         uint32_t xo_remote, xml_remote;
-        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(xo_remote) : "r"(xo_local));
-        asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(xml_remote) : "r"(xml_local));
+        const uint32_t peer = (uint32_t)(split ^ 1);
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xo_remote) : "r"(xo_local), "r"(peer));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(xml_remote) : "r"(xml_local), "r"(peer));
 #pragma unroll 1
         for (int c0 = 0; c0 < kPartCols; c0 += 32) {
           float o[32];
@@ -377,8 +381,8 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (part == 0)
           asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(xml_remote), "f"(m), "f"(l_row) : "memory");
       }
-      pair_sync();                                              // the second split's numbers have landed
-      if (split == 0) {
+      pair_sync();                                              // the partner's numbers have landed
+      if (mine) {
         float m1, l1;
         asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(m1), "=f"(l1) : "r"(xml_local) : "memory");
         const bool has0 = l_row > 0.f, has1 = l1 > 0.f;
