@@ -319,25 +319,27 @@ cross_topk_kernel(const uint32_t* __restrict__ ckey_all, const int32_t* __restri
 // Gather for a free-form ascending unit list (same length S_u for every slab, any split between contexts).
 // Unit at list position p lands at slot p*B - (tokens missing from the short tail units of earlier contexts).
 // ---------------------------------------------------------------------------------------------
+constexpr int kUnitCopyThreads = 128, kUnitCopyRows = 32;    // small CTAs: they share SMs with attention CTAs
+
 template <int kRowBytes>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kUnitCopyThreads)
 compact_units_kernel(const char* __restrict__ K, const char* __restrict__ V, const int32_t* __restrict__ sel,
                      char* __restrict__ Kc, char* __restrict__ Vc, int32_t* __restrict__ cache_len,
                      int32_t* __restrict__ inv_map, const __grid_constant__ CtxTable ct,
                      const __grid_constant__ TopTable tt, int Hkv, int L_tot, int S_u, int S, int capacity, int chunks,
                      int* __restrict__ d_status) {
   constexpr int kLanes = kRowBytes / 16;
-  constexpr int kRowsPerPass = 256 / kLanes;
-  constexpr int kPasses = 64 / kRowsPerPass;
+  constexpr int kRowsPerPass = kUnitCopyThreads / kLanes;
+  constexpr int kPasses = kUnitCopyRows / kRowsPerPass;
   const int chunk = blockIdx.x % chunks;
   const size_t slab = blockIdx.x / chunks;
   const int lane = threadIdx.x % kLanes, rsub = threadIdx.x / kLanes;
   if (chunk == 0 && threadIdx.x == 0 && (slab % Hkv) == 0) cache_len[slab / Hkv] = S;
   const int B = ct.block_size;
   // virtual row (list position * B + offset in unit) -> (source token, slot), once per row of the CTA
-  __shared__ int s_tok[64], s_slot[64];
-  if (threadIdx.x < 64) {
-    const int v = chunk * 64 + threadIdx.x;
+  __shared__ int s_tok[kUnitCopyRows], s_slot[kUnitCopyRows];
+  if (threadIdx.x < kUnitCopyRows) {
+    const int v = chunk * kUnitCopyRows + threadIdx.x;
     int t = -1, slot = -1;
     if (v < S_u * B) {
       const int pos = v >> ct.block_shift, j = v & (B - 1);
@@ -456,12 +458,12 @@ cudaError_t launch_compact_units(const samkv_shape_t& s, const CtxTable& ct, con
     if (e != cudaSuccess) return e;
   }
   const int rows = S_u * ct.block_size;
-  const int chunks = rows > 0 ? (rows + 63) / 64 : 1;
+  const int chunks = rows > 0 ? (rows + kUnitCopyRows - 1) / kUnitCopyRows : 1;
   const long long blocks = slabs * chunks;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   const int row_bytes = s.head_dim * (s.dtype == SAMKV_BF16 ? 2 : 4);
 #define SAMKV_LAUNCH_CU(RB)                                                                                         \
-  compact_units_kernel<RB><<<(unsigned)blocks, 256, 0, stream>>>((const char*)K, (const char*)V, sel, (char*)Kc,     \
+  compact_units_kernel<RB><<<(unsigned)blocks, kUnitCopyThreads, 0, stream>>>((const char*)K, (const char*)V, sel, (char*)Kc,     \
                                                                  (char*)Vc, cache_len, inv_map, ct, tt, s.n_kv_heads, \
                                                                  L_tot, S_u, S, capacity, chunks, d_status)
   switch (row_bytes) {
