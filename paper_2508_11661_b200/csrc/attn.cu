@@ -92,6 +92,7 @@ __global__ void append_kernel(char* __restrict__ Kc, char* __restrict__ Vc, cons
                               const char* __restrict__ Kq, const char* __restrict__ Vq, int Hkv, int T_q, int capacity,
                               int row_bytes, long long n_threads, int* __restrict__ d_status) {
   pdl_launch_dependents();      // the attention kernel may set itself up while the chunk is being appended
+  pdl_wait();                   // the kernel before this one may be the previous call's attention: it bumps cache_len
   const int lanes = row_bytes / 16;
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= n_threads) return;
@@ -319,9 +320,21 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   if (appended) {
     const int row_bytes = kHeadDim * (int)sizeof(T);
     const long long threads = (long long)Bt * T_q * Hkv * (row_bytes / 16);
-    append_kernel<<<(unsigned)((threads + 127) / 128), 128, 0, stream>>>((char*)Kl, (char*)Vl, len_l, (const char*)Kq,
-                                                                        (const char*)Vq, Hkv, T_q, capacity, row_bytes,
-                                                                        threads, d_status);
+    // launched as a programmatic dependent: it is scheduled when the kernel before it in the stream releases its
+    // dependents (the attention kernels do so once their results are written) and waits for that kernel's completion
+    // before it reads cache_len, so only the launch latency overlaps
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((threads + 127) / 128));
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, append_kernel, (char*)Kl, (char*)Vl, (const int32_t*)len_l, (const char*)Kq,
+                                       (const char*)Vq, Hkv, T_q, capacity, row_bytes, threads, d_status);
+    if (e != cudaSuccess) return e;
   }
   const int G = Hq / Hkv;
   const int rows = T_q * G;
