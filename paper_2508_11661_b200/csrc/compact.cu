@@ -6,8 +6,8 @@
 
 namespace samkv {
 
-constexpr int kCopyThreads = 128;
-constexpr int kCompactRowsPerCta = 32;
+constexpr int kCopyThreads = 64;
+constexpr int kCompactRowsPerCta = 8;
 
 template <int kRowBytes>
 __global__ void __launch_bounds__(kCopyThreads)

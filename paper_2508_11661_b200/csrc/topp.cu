@@ -319,7 +319,7 @@ cross_topk_kernel(const uint32_t* __restrict__ ckey_all, const int32_t* __restri
 // Gather for a free-form ascending unit list (same length S_u for every slab, any split between contexts).
 // Unit at list position p lands at slot p*B - (tokens missing from the short tail units of earlier contexts).
 // ---------------------------------------------------------------------------------------------
-constexpr int kUnitCopyThreads = 128, kUnitCopyRows = 32;    // small CTAs: they share SMs with attention CTAs
+constexpr int kUnitCopyThreads = 64, kUnitCopyRows = 8;    // small CTAs: they share SMs with attention CTAs
 
 template <int kRowBytes>
 __global__ void __launch_bounds__(kUnitCopyThreads)
