@@ -245,7 +245,7 @@ samkv_status_t samkv_compact_units(samkv_handle_t h, const samkv_shape_t* shape,
 int32_t samkv_attn_kernel_count(samkv_handle_t h, const samkv_shape_t* shape, int32_t T_q, int32_t cache_capacity,
                                 int32_t appended);
 
-/* ---- block representatives (Sec. 3.2: "each block is represented by the mean vector of its token caches") --- */
+/* ---- block representatives (Sec. 3.2: a block's representative is the mean of its tokens' keys) ------------ */
 
 /* Kbar[l,b,h,u,:] = mean over the tokens of unit u of K[l,b,h,t,:] (fp32 sum in a fixed order, one rounding to the
  * storage dtype; a short tail unit averages the tokens it has).  Query-independent: run once per stored document.
@@ -305,6 +305,10 @@ samkv_status_t samkv_align(samkv_handle_t h, const samkv_shape_t* shape, const i
  *     call's contents; every element a call reads is rewritten by that call first, so no clearing
  *     is needed.
  *   - Calls no cudaMalloc / cudaFree or any other allocating routine.
+ *   - There is no handle and therefore no status word: a device-side check that samkv_score would record for
+ *     samkv_poll_status (a bounded wait inside the scoring kernel that ran out) is NOT reported by this entry
+ *     point.  The kernel still gives up and returns, part of scores_out is then left unwritten, and the call
+ *     has long returned SAMKV_OK.  A caller that needs that report uses samkv_score with a workspace.
  * Arguments as in samkv_score (K, Q, Qloc, scores_out are caller-owned device pointers). */
 #define SAMKV_STATIC_SCORE_MAX_FLOATS (256 * 1024)
 samkv_status_t samkv_score_static(const samkv_shape_t* shape, const void* K, const void* Q, int32_t T_q,

@@ -91,7 +91,7 @@ samkv_status_t make_sel_table(const samkv_shape_t* s, const Layout& lo, const in
     int toks = k * s->block_size;
     if (lo.tail[c] != s->block_size && k > 0) toks -= s->block_size - lo.tail[c];
     st->slot_off[c + 1] = st->slot_off[c] + toks;
-    st->n_init_units[c] = (short)lo.n_init_units[c];
+    st->n_init_units[c] = lo.n_init_units[c];
     st->first_local_unit[c] = lo.first_local_unit[c];
   }
   *S = st->slot_off[s->n_ctx];

@@ -29,10 +29,7 @@ using namespace tc;
 
 constexpr int kBM = 128, kBN = 128, kD = 128;
 constexpr int kStagesK = 3, kStagesV = 2;
-#ifndef SAMKV_TC3_PARTS
-#define SAMKV_TC3_PARTS 2
-#endif
-constexpr int kParts = SAMKV_TC3_PARTS;       // threads per row: each owns kPartCols score columns and O columns
+constexpr int kParts = 2;                     // threads per row: each owns kPartCols score columns and O columns
 constexpr int kPartCols = kBN / kParts;
 constexpr int kSoftmaxWarps = 4 * kParts;
 constexpr int kMmaWarp = kSoftmaxWarps, kLoadWarp = kSoftmaxWarps + 1;

@@ -22,7 +22,7 @@ struct CtxTable {
 struct SelTable {
   int sel_off[SAMKV_MAX_CTX + 1];       // prefix sum of k_units
   int slot_off[SAMKV_MAX_CTX + 1];      // prefix sum of kept tokens
-  short n_init_units[SAMKV_MAX_CTX];    // protected units at the start of the context
+  int n_init_units[SAMKV_MAX_CTX];      // protected units at the start of the context
   int first_local_unit[SAMKV_MAX_CTX];  // first unit protected because it overlaps the last n_local tokens
 };
 

@@ -4,8 +4,8 @@ device synchronisation is unacceptable).  Its scratch is a fixed array inside th
 handle and no workspace.  Checked here, through the C ABI, against the regular samkv_score on two calls
 in a row (the second with other inputs, so that stale scratch contents would show), plus the size limit.
 
-This file is named to be collected last: a run that stops at the first failure has then already run
-every other test.
+The entry point keeps state inside the library (the fixed array and its cached address), so this file sorts
+after the other test files and runs once they have finished.
 """
 import ctypes
 
