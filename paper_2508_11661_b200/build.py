@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsamkv.so")
-SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "topp.cu", "align.cu", "means.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu", "attn_tc3.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "topp.cu", "align.cu", "means.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu", "attn_tc4.cu"]
 
 
 def nvcc_path() -> str:

@@ -23,7 +23,7 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
                             cudaStream_t stream);
-cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
+cudaError_t launch_attn_tc4(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
                             const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
                             float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
 
@@ -35,12 +35,15 @@ cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* 
 // plus `fixed_cost` for its prologue and epilogue (any common unit).  A grid that spills a few CTAs into one more
 // wave costs a whole wave.
 static long long best_split(long long base_ctas, long long tiles, long long slots, long long max_splits,
-                            long long tile_cost, long long fixed_cost, long long* cost_out) {
+                            long long tile_cost, long long fixed_cost, long long* cost_out,
+                            long long fixed_cost_3plus = -1) {
   long long best_n = 1, best_cost = -1;
   for (long long n = 1; n <= max_splits; ++n) {
     const long long tps = (tiles + n - 1) / n;
     const long long waves = (base_ctas * n + slots - 1) / slots;
-    const long long cost = waves * (tps * tile_cost + fixed_cost);
+    // (a kernel that merges one or two splits itself pays more once partial results go through global memory)
+    const long long fixed = (n >= 3 && fixed_cost_3plus >= 0) ? fixed_cost_3plus : fixed_cost;
+    const long long cost = waves * (tps * tile_cost + fixed);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
   }
   *cost_out = best_cost;
@@ -59,12 +62,13 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
   long long cost = 0;
   if (s.dtype == SAMKV_BF16 && rows >= 128 && s.head_dim == 128) {
     // The two tcgen05 kernels, one CTA per SM, 128-slot tiles.  Measured on B200 (cycles): 256 rows per CTA
-    // (two query tiles share every K/V tile) ~5000 per tile + ~20000 per CTA; 128 rows per CTA (score tile
-    // double-buffered) ~2760 per tile + ~9000 per CTA.  Short KV ranges favour the second, long ones the first.
+    // (two query tiles share every K/V tile, which halves the L2 traffic) ~4070 per tile + ~35000 per CTA;
+    // 128 rows per CTA (two groups of tiles taking turns) ~2150 per tile + ~8000 per CTA (~22000 with three or more splits, which go through global memory).  The second wins
+    // everywhere except on very long KV ranges.
     const long long tiles = (capacity + 127) / 128;
     long long cost256 = 0, cost128 = 0;
-    const long long n256 = best_split(bh * ((rows + 255) / 256), tiles, sm_count, max_splits, 5000, 20000, &cost256);
-    const long long n128 = best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2760, 9000, &cost128);
+    const long long n256 = best_split(bh * ((rows + 255) / 256), tiles, sm_count, max_splits, 4070, 35000, &cost256);
+    const long long n128 = best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2150, 8000, &cost128, 22000);
     const bool use128 = cost128 <= cost256;
     p.rows_per_cta = use128 ? 128 : 256;
     p.n_splits = (int)(use128 ? n128 : n256);
@@ -340,7 +344,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
     cudaError_t e = (plan.rows_per_cta == 128)
-                        ? launch_attn_tc3(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                        ? launch_attn_tc4(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
                                           plan, d_status, stream)
                     : (plan.rows_per_cta == 256)
                         ? launch_attn_tc2(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
@@ -356,7 +360,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
         Kl, Vl, len_l, (const T*)Q, (T*)O, lse, part_o, part_ml, Hq, Hkv, T_q, capacity, appended, scale,
         plan.n_splits, row_tiles);
   }
-  if ((plan.n_splits > 1 || appended) && !(sizeof(T) == 2 && attn_tc3_merges_in_cluster(plan))) {
+  if ((plan.n_splits > 1 || appended) && !(sizeof(T) == 2 && attn_merges_in_cluster(plan))) {
     const long long blocks = plan.n_splits > 1 ? (long long)((out_rows + 3) / 4) : 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);

@@ -74,7 +74,7 @@ struct AttnPlan {
 };
 AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count);
 // The 128-row tcgen05 kernel with exactly two KV splits merges them inside a two-CTA cluster: no merge kernel.
-inline bool attn_tc3_merges_in_cluster(const AttnPlan& p) { return p.rows_per_cta == 128 && p.n_splits == 2; }
+inline bool attn_merges_in_cluster(const AttnPlan& p) { return p.rows_per_cta == 128 && p.n_splits == 2; }
 // Status block of the workspace (256 bytes, zero between calls): int 0 is the device check word, this int counts the
 // finished CTAs of an attention grid that bumps cache_len itself.
 constexpr int kAttnTicketInt = 32;

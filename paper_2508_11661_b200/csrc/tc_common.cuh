@@ -13,7 +13,11 @@ namespace tc {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
-constexpr uint32_t kSpinLimit = 1u << 22;
+#ifdef SAMKV_TC_SPIN_LIMIT
+constexpr uint32_t kSpinLimit = SAMKV_TC_SPIN_LIMIT;
+#else
+constexpr uint32_t kSpinLimit = 1u << 20;
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
@@ -38,7 +42,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
+#ifdef SAMKV_TC_TEST_WAIT
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#else
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
@@ -50,7 +58,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // Whole-warp wait: one lane polls, the rest park at the warp barrier, which keeps barrier traffic out of
 // the shared-memory pipeline that the tensor core's operand reads already saturate.
 __device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* s_fail) {
+#ifdef SAMKV_TC_ALL_LANES_POLL
+  mbar_wait(bar, parity, s_fail);
+#else
   if ((threadIdx.x & 31) == 0) mbar_wait(bar, parity, s_fail);
+#endif
   __syncwarp();
 }
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
