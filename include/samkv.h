@@ -18,6 +18,11 @@
  *   - Calls validate their arguments on the host, then only enqueue kernels on `stream`
  *     (a cudaStream_t passed as void*; NULL = the default stream).  They do not allocate,
  *     free or synchronise (samkv_poll_status is the one call that synchronises).
+ *   - Plain stream order holds for every argument: whatever earlier work on `stream` wrote (Q
+ *     from a projection kernel, the cache from samkv_update, cache_len from the previous call)
+ *     is seen by the call.  Some kernels are launched so that their set-up overlaps the tail of
+ *     the kernel before them (programmatic dependent launch); they read nothing the caller
+ *     passes before that kernel has completed.
  *   - A handle owns no memory: scratch lives in the caller's `workspace`.  Calls that use the
  *     same handle must be ordered on one stream (they share the workspace).
  *   - On a host-detected error a call returns a non-zero status and launches nothing.

@@ -363,7 +363,8 @@ int32_t samkv_attn_kernel_count(samkv_handle_t handle, const samkv_shape_t* shap
   if (h == nullptr || make_layout(shape, &lo) != SAMKV_OK || T_q < 1 || cache_capacity < 1) return 0;
   const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count);
   const bool self_merge = shape->dtype == SAMKV_BF16 && attn_merges_in_cluster(plan);
-  int n = 1 + (appended ? 1 : 0);
+  const bool self_append = shape->dtype == SAMKV_BF16 && shape->head_dim == 128 && plan.rows_per_cta == 128;
+  int n = 1 + ((appended && !self_append) ? 1 : 0);
   if ((plan.n_splits > 1 || appended) && !self_merge) ++n;
   return n;
 }

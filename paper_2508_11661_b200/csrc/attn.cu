@@ -23,9 +23,9 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
                             cudaStream_t stream);
-cudaError_t launch_attn_tc4(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
-                            const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
-                            float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
+cudaError_t launch_attn_tc4(const samkv_shape_t& s, void* Kc, void* Vc, int capacity, int32_t* cache_len,
+                            const void* Q, int T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
+                            float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------------
 // Plan: how many packed rows a CTA takes and into how many KV splits a (batch, kv head) is cut.
@@ -321,7 +321,9 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   float* part_o = (float*)partial_ws;
   float2* part_ml = (float2*)(part_o + out_rows * plan.n_splits * kHeadDim);
 
-  if (appended) {
+  // the 128-row tensor-memory kernel writes the chunk's rows into the cache itself
+  const bool self_append = sizeof(T) == 2 && kHeadDim == 128 && plan.rows_per_cta == 128;
+  if (appended && !self_append) {
     const int row_bytes = kHeadDim * (int)sizeof(T);
     const long long threads = (long long)Bt * T_q * Hkv * (row_bytes / 16);
     // launched as a programmatic dependent: it is scheduled when the kernel before it in the stream releases its
@@ -344,7 +346,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
     cudaError_t e = (plan.rows_per_cta == 128)
-                        ? launch_attn_tc4(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                        ? launch_attn_tc4(s, Kl, Vl, capacity, len_l, Q, T_q, Kq, Vq, scale, O, lse, part_o, part_ml,
                                           plan, d_status, stream)
                     : (plan.rows_per_cta == 256)
                         ? launch_attn_tc2(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,

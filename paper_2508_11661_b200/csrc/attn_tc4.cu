@@ -19,6 +19,10 @@
 //               commit costs it 100-300 cycles, which the other issuer's products cover.
 //   warp 10     loader: K and V tiles (3 stages each) arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle)
 //   warp 11     idle: it completes the third warpgroup, which hands registers to the softmax warps (setmaxnreg)
+// The chunk's own K/V rows (the "append" of the incremental prefill) are written into the cache by this kernel: every
+// CTA whose KV range reaches past cache_len copies the rows of its (batch, kv head) itself before its loader fetches
+// those tiles.  Several CTAs then write the same bytes to the same addresses, which is harmless and needs no
+// dependency between CTAs.
 // Tensor memory: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_g overlays the first 64 columns of S_g.
 // Barriers are indexed by tile number mod 6 (a multiple of the group count 2 and the stage count 3), so that no
 // waiter can be a whole round behind.
@@ -65,7 +69,9 @@ enum Bar {
   FULL = kRound,      // S(t) is complete, and so is O += P(t-2) V(t-2): the group may read S(t) and touch O; K stage of
                       // tile t and V stage of tile t-2 are free
   K01 = 2 * kRound,   // K(0), K(1) have landed (two slots)
-  KV_TMA = 2 * kRound + 2, O_FINAL /* two slots */, Q_READY = O_FINAL + 2, N_BARS
+  KV_TMA = 2 * kRound + 2, O_FINAL /* two slots */, Q_READY = O_FINAL + 2,
+  APPENDED,           // this CTA's copy of the chunk's K/V rows into the cache is complete (8 softmax warps)
+  N_BARS
 };
 
 // two fp32 values in one 64-bit register, for the packed fp32 instructions
@@ -92,16 +98,20 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-// Two positive finite fp32 values -> packed bf16 (lo in the low half), rounded to nearest with ties away from zero:
+// Two non-negative finite fp32 values -> packed bf16 (lo in the low half), rounded to nearest with ties away from zero:
 // 0x8000 is added to the bit patterns and one byte permute takes the upper halves.  This keeps the conversion off the
 // special-function pipe, where cvt.rn.bf16x2.f32 runs at a quarter of the rate next to the exponentials.  (The
-// probabilities are <= 2^65 here, so the increment cannot carry into an infinity.)
-__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
+// probabilities are <= 2^65 here, so the increment cannot carry into an infinity.)  lo and hi are replaced by the
+// rounded values: the row sum is taken over exactly what the tensor core multiplies with V, so that the rounding of
+// a dominant probability cancels between numerator and denominator instead of showing up in the output.
+__device__ __forceinline__ uint32_t round_pack_bf16(float& lo, float& hi) {
+  const uint32_t a = __float_as_uint(lo) + 0x8000u, b = __float_as_uint(hi) + 0x8000u;
   uint32_t r;
-  asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(r) : "r"(__float_as_uint(lo) + 0x8000u), "r"(__float_as_uint(hi) + 0x8000u));
+  asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(r) : "r"(a), "r"(b));
+  lo = __uint_as_float(a & 0xffff0000u);
+  hi = __uint_as_float(b & 0xffff0000u);
   return r;
 }
-
 
 }  // namespace tc4
 
@@ -112,11 +122,13 @@ __device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
 template <bool kPair>
 __global__ void __launch_bounds__(tc4::kThreads, 1)
 attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                int32_t* cache_len, const __nv_bfloat16* __restrict__ Q,
+                int32_t* cache_len, const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ Kq,
+                const __nv_bfloat16* __restrict__ Vq, __nv_bfloat16* Kc, __nv_bfloat16* Vc,
                 __nv_bfloat16* __restrict__ O, float* __restrict__ lse, float* __restrict__ part_o,
-                float2* __restrict__ part_ml, int Hq, int Hkv, int T_q, int capacity, int appended, float scale,
+                float2* __restrict__ part_ml, int Hq, int Hkv, int T_q, int capacity, float scale,
                 int n_splits, int row_tiles, int* __restrict__ d_status) {
   using namespace tc4;
+  const int appended = Kq != nullptr;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   // A misaligned buffer (never seen: the declaration asks for 1024 bytes) is reported and the CTA does no tile work,
@@ -154,6 +166,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     mbar_init(bar(O_FINAL), 1);
     mbar_init(bar(O_FINAL + 1), 1);
     mbar_init(bar(Q_READY), kSoftmaxWarps);
+    mbar_init(bar(APPENDED), kSoftmaxWarps);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -194,8 +207,40 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const int tile0 = split * tps;
   const int tile1 = min(min(tile0 + tps, n_tiles), (cta_visible + kBN - 1) / kBN);
   const int nt = bad_smem ? 0 : max(tile1 - tile0, 0);
+  // The chunk's own K/V rows belong at slots len .. len + T_q - 1 of the cache.  Every CTA whose KV range reaches
+  // past `len` writes them there itself before its loader fetches those tiles (several CTAs write the same bytes to
+  // the same addresses: harmless), so no separate kernel and no dependency between CTAs is needed.  The CTA of the
+  // last row tile and last split always does, so the rows are in the cache when the call completes.
+  const bool copies_chunk = n_app > 0 && ((tile0 + nt) * kBN > len || (rtile == row_tiles - 1 && split == n_splits - 1));
+  if (appended && n_app == 0 && blockIdx.x == 0 && tid == 0) atomicMax(d_status, (int)CHECK_APPEND_CAPACITY);
 
   if (warp < kSoftmaxWarps) {
+    if (copies_chunk) {
+      for (int i0 = 0; i0 < T_q * 16; i0 += kSoftmaxWarps * 32 * 4) {      // four rows' pieces in flight per thread
+        uint4 vk[4], vv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kSoftmaxWarps * 32 + tid;
+          if (i < T_q * 16) {
+            const size_t src = (((size_t)b * T_q + (i >> 4)) * Hkv + h) * kD + (i & 15) * 8;
+            vk[u] = ld_stream(Kq + src);
+            vv[u] = ld_stream(Vq + src);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kSoftmaxWarps * 32 + tid;
+          if (i < T_q * 16) {
+            const size_t dst = ((size_t)bh * capacity + len + (i >> 4)) * kD + (i & 15) * 8;
+            *reinterpret_cast<uint4*>(Kc + dst) = vk[u];
+            *reinterpret_cast<uint4*>(Vc + dst) = vv[u];
+          }
+        }
+      }
+      asm volatile("fence.proxy.async;" ::: "memory");          // the TMA loads of this CTA must see these rows
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(APPENDED));
+    }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     fence_proxy_async();
     __syncwarp();
@@ -215,7 +260,15 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       tma_load_3d(dst, map, 0, j0, bh, target);
       tma_load_3d(dst + kBN * 128, map, 64, j0, bh, target);
     };
+    bool chunk_in_cache = !copies_chunk;
+    auto before_tile = [&](int t) {                               // a tile that reaches past `len` holds rows of the chunk
+      if (!chunk_in_cache && (tile0 + t) * kBN + kBN > len) {
+        wait(APPENDED, 0);
+        chunk_in_cache = true;
+      }
+    };
     for (int t = 0; t < 2 && t < nt; ++t) {
+      before_tile(t);
       if (lane == 0) {
         mbar_expect_tx(bar(K01 + t), kTileBytes);
         load_tile(&tmK, sK + t * kTileBytes, t, bar(K01 + t));
@@ -227,6 +280,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       if (t >= 1) wait(FULL + (t - 1) % kRound, (uint32_t)((t - 1) / kRound));
       const uint32_t sv = sV + (t % kStages) * kTileBytes;
       const bool with_k = t + 2 < nt;
+      before_tile(with_k ? t + 2 : t);
       const bool partial = (tile0 + t) * kBN + kBN > total;      // V rows past `total` must read as zero
       if (lane == 0) {
         const uint32_t target = partial ? bar(KV_TMA) : bar(GO + t % kRound);
@@ -362,9 +416,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         for (int i = 0; i < 16; ++i) {
           float x0, x1;
           unpack2(fma2(pack2(sv[c0 + 2 * i], sv[c0 + 2 * i + 1]), sl2_2, negmu2), x0, x1);
-          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+          float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+          pk[i] = round_pack_bf16(p0, p1);
           if (i & 1) psb = add2(psb, pack2(p0, p1)); else psa = add2(psa, pack2(p0, p1));
-          pk[i] = pack_bf16_int(p0, p1);
         }
         tmem_st16(tS + (c0 >> 1), pk);
       };
@@ -559,9 +613,9 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   }
 }
 
-cudaError_t launch_attn_tc4(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
-                            const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
-                            float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream) {
+cudaError_t launch_attn_tc4(const samkv_shape_t& s, void* Kc, void* Vc, int capacity, int32_t* cache_len,
+                            const void* Q, int T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
+                            float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream) {
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = T_q * G;
   const int row_tiles = (rows + tc4::kBM - 1) / tc4::kBM;
@@ -575,8 +629,8 @@ cudaError_t launch_attn_tc4(const samkv_shape_t& s, const void* Kc, const void* 
   auto kern = pair ? attn_tc4_kernel<true> : attn_tc4_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc4::kSmemBytes);
   if (e != cudaSuccess) return e;
-  // Launched so that it may start while the kernel before it in the stream (the append of the chunk) is still
-  // running: barrier set-up and the tensor-memory allocation need nothing from it; one wait precedes every read.
+  // Launched so that it may start while the kernel before it in the stream is still running: barrier set-up and the
+  // tensor-memory allocation need nothing from it; one wait precedes every read.
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)blocks);
   cfg.blockDim = dim3(tc4::kThreads);
@@ -591,9 +645,9 @@ cudaError_t launch_attn_tc4(const samkv_shape_t& s, const void* Kc, const void* 
   attrs[1].val.clusterDim.z = 1;
   cfg.attrs = attrs;
   cfg.numAttrs = pair ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, kern, tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (__nv_bfloat16*)O, lse, part_o,
-                            part_ml, s.n_q_heads, s.n_kv_heads, T_q, capacity, appended, scale, plan.n_splits, row_tiles,
-                            d_status);
+  return cudaLaunchKernelEx(&cfg, kern, tmK, tmV, cache_len, (const __nv_bfloat16*)Q, (const __nv_bfloat16*)Kq,
+                            (const __nv_bfloat16*)Vq, (__nv_bfloat16*)Kc, (__nv_bfloat16*)Vc, (__nv_bfloat16*)O, lse, part_o,
+                            part_ml, s.n_q_heads, s.n_kv_heads, T_q, capacity, scale, plan.n_splits, row_tiles, d_status);
 }
 
 }  // namespace samkv

@@ -202,6 +202,18 @@ def attn_tolerance(w) -> float:
     return 2e-2 if w.dtype == "bf16" else 1e-4
 
 
+# The absolute bf16 bound is loose where the outputs are small (with N(0,1) values and thousands of visible slots
+# |O| is a few hundredths), so a second, relative bound goes with it: per query head, the largest error may be at
+# most 2^-6 of the largest oracle output of that head.  The kernels round P and O to bf16 (2^-9 relative each) and
+# accumulate in fp32, so errors of about 2^-8 of the head's largest output are expected; 2^-6 leaves a factor of
+# four and still fails a result that is off by a few percent.  The softmax denominator is summed in fp32 over the
+# bf16-rounded probabilities (the values the tensor core multiplies with V), so lse can be off by log(1 + 2^-9) =
+# 2e-3 when one probability dominates; its bound is 2^-8.
+ATTN_REL_BOUND_BF16 = 2.0 ** -6
+LSE_BOUND_BF16 = 2.0 ** -8
+OBSERVED = {"attn_rel": 0.0, "lse": 0.0}      # largest values seen in this process (printed by the tests that ask)
+
+
 def check_attention(w, Kc_lb, Vc_lb, cache_len, Q_b, Kq_b, Vq_b, O_gpu_b, lse_gpu_b=None, scale=None, t_sample=None):
     """Oracle attention on the GPU's own compact cache values; optional sampling of query tokens
     (only when nothing is appended, so that visibility does not depend on the token index)."""
@@ -217,9 +229,19 @@ def check_attention(w, Kc_lb, Vc_lb, cache_len, Q_b, Kq_b, Vq_b, O_gpu_b, lse_gp
         got = got[t_sample]
     err = np.abs(got - out).max()
     assert err <= attn_tolerance(w), f"attention max-abs error {err}"
+    if w.dtype == "bf16":
+        # out, got: [T, Hq, d] -> per query head over tokens and elements
+        head_err = np.abs(got - out).max(axis=(0, 2))
+        head_max = np.abs(out).max(axis=(0, 2))
+        rel = float((head_err / np.maximum(head_max, 1e-30)).max())
+        OBSERVED["attn_rel"] = max(OBSERVED["attn_rel"], rel)
+        assert rel <= ATTN_REL_BOUND_BF16, f"attention error {rel:.3e} of a head's largest output (bound 2^-6)"
     if lse_gpu_b is not None:
         lg = to_f64(lse_gpu_b)
         if t_sample is not None:
             lg = lg[:, t_sample]
-        assert np.abs(lg - lse).max() <= (2e-2 if w.dtype == "bf16" else 1e-4)
+        lse_err = float(np.abs(lg - lse).max())
+        if w.dtype == "bf16":
+            OBSERVED["lse"] = max(OBSERVED["lse"], lse_err)
+        assert lse_err <= (LSE_BOUND_BF16 if w.dtype == "bf16" else 1e-4), f"lse error {lse_err}"
     return err, K2, V2, n

@@ -179,7 +179,11 @@ def test_cfg2_timed_schedule_matches_in_order_and_oracle():
     assert torch.equal(pipe.O.view(torch.int16), ref["O"].view(torch.int16))
     assert int(pipe.cache_len[0, 0]) == pipe.S + w.q_tokens
     inp = pipe.inp
-    for (l, b) in [(0, 0), (13, 1), (31, 3)]:
+    rng = np.random.default_rng(2026)                    # eight (layer, batch element) problems by a seeded draw
+    picks = {(0, 0), (31, 3)}
+    while len(picks) < 8:
+        picks.add((int(rng.integers(w.n_layers)), int(rng.integers(w.batch))))
+    for (l, b) in sorted(picks):
         check_attention(w, pipe.Kc[l, b], pipe.Vc[l, b], pipe.S, inp["Qa"][l, b], inp["Kq"][l, b], inp["Vq"][l, b],
                         pipe.O[l, b])
     del pipe, ref

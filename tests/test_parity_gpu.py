@@ -365,6 +365,62 @@ def test_chunked_prefill_on_the_tensor_memory_kernel():
         assert np.array_equal(to_f64(run.Kc[0, b])[:, :n], Kc_ref[b][:, :n])
 
 
+def test_attention_sees_q_written_by_the_kernel_right_before_it():
+    """Stream order on Q: a kernel on the same stream writes Q immediately before every one of several hundred
+    back-to-back attention calls on the tensor-memory path (which is launched as a programmatic dependent and
+    overlaps its set-up with the kernel before it).  Every output must equal the output for that Q computed after
+    a full synchronisation, and those reference outputs are checked against the oracle."""
+    w = synth.CONFIGS["cfg1"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = DeviceRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    g = torch.Generator(device=DEV).manual_seed(5)
+    n_src, n_calls = 4, 320
+    Q_src = torch.randn((n_src,) + tuple(inp["Qa"][0].shape), generator=g, device=DEV).to(w.torch_dtype)
+    Kc0, Vc0 = run.Kc[0].clone(), run.Vc[0].clone()
+    for with_chunk in (False, True):
+        Kq = inp["Kq"][0] if with_chunk else None
+        Vq = inp["Vq"][0] if with_chunk else None
+        refs = []
+        for i in range(n_src):                                # references: everything complete before the call
+            run.cache_len.fill_(run.S)
+            torch.cuda.synchronize()
+            Oref, lse = run.attn(0, Q_src[i].clone(), Kq, Vq)
+            torch.cuda.synchronize()
+            check_attention(w, Kc0[0], Vc0[0], run.S, Q_src[i][0], None if Kq is None else Kq[0],
+                            None if Vq is None else Vq[0], Oref[0], lse[0])
+            refs.append(Oref)
+        Q = torch.empty_like(Q_src[0])
+        outs = torch.empty((n_calls,) + tuple(Q.shape), dtype=Q.dtype, device=DEV)
+        for i in range(n_calls):                              # no host synchronisation in this loop
+            if with_chunk:
+                run.cache_len.fill_(run.S)
+            Q.copy_(Q_src[i % n_src])                         # the producer of Q: a kernel on the same stream
+            B.samkv_attn(run.handle, run.shape, 0, run.Kc, run.Vc, run.capacity, run.cache_len, Q, w.q_tokens, Kq, Vq,
+                         0.0, outs[i], None)
+        torch.cuda.synchronize()
+        assert run.poll() == 0
+        for i in range(n_calls):
+            assert torch.equal(outs[i], refs[i % n_src]), f"call {i} (chunk appended: {with_chunk}) read a stale Q"
+
+
+def test_a_five_percent_error_in_attention_would_be_caught():
+    """The relative bound bites on N(0,1) data: the library's own cfg1 output, scaled by 1.05, fails it."""
+    import samkv_testlib as T
+    w = synth.CONFIGS["cfg1"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = DeviceRun(w, inp).sparsify()
+    Kc0, Vc0 = run.Kc[0].clone(), run.Vc[0].clone()
+    Og, lse = run.attn(0, inp["Qa"][0], inp["Kq"][0], inp["Vq"][0])
+    torch.cuda.synchronize()
+    T.OBSERVED["attn_rel"] = 0.0
+    check_attention(w, Kc0[0], Vc0[0], run.S, inp["Qa"][0, 0], inp["Kq"][0, 0], inp["Vq"][0, 0], Og[0], lse[0])
+    print(f"cfg1 attention: largest error {T.OBSERVED['attn_rel']:.3e} of a head's largest output, lse {T.OBSERVED['lse']:.3e}")
+    with pytest.raises(AssertionError):
+        check_attention(w, Kc0[0], Vc0[0], run.S, inp["Qa"][0, 0], inp["Kq"][0, 0], inp["Vq"][0, 0],
+                        (Og[0].float() * 1.05).to(Og.dtype), lse[0])
+
+
 @pytest.mark.parametrize("ctx_lens,T_q,Hq,Hkv,budget_bp", [
     ((40, 30), 32, 8, 2, 10000),          # 128 rows, one partial KV tile: cache (70) + chunk (32) < 128 slots
     ((100, 90), 129, 2, 2, 10000),        # G = 1, 129 rows: a second query tile with a single real row
