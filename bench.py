@@ -37,11 +37,19 @@ HBM_NOMINAL_GBS = 8000.0
 HBM_FALLBACK_GBS = 6650.0
 
 # kernels each C-ABI call enqueues (memsets are not counted)
-# DRAM bytes per scored key row of score_stream_kernel, from the ncu capture summarised in
-# profiles/score_stream_kernel_cfg2_2layers.md (dram read + write of one launch / rows of that launch);
-# traffic grows in proportion to the rows (no reuse), so a full launch is rows x this figure.
-SCORE_KERNEL_DRAM_BYTES_PER_ROW = 260.0
 KERNELS_PER_CALL = {"score": 2, "select": 1, "compact": 1, "update": 1}      # samkv_attn: asked from the library
+
+
+def score_kernel_dram_bytes_per_row():
+    """DRAM bytes per scored key row of score_stream_kernel (dram read + write of one launch / rows of that launch),
+    from the ncu capture summarised under profiles/; traffic grows in proportion to the rows (no reuse), so a full
+    launch is rows x this figure.  Kept in a small file beside the profile it came from."""
+    p = os.path.join(ROOT, "profiles", "score_stream_kernel_dram_bytes.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["dram_bytes_per_row"])
+    except Exception:
+        return None
 
 
 def measured_peaks():
@@ -55,14 +63,20 @@ def measured_peaks():
 # --------------------------------------------------------------------------------------------------
 # algorithmic bytes of one step (what the method itself must move)
 # --------------------------------------------------------------------------------------------------
-def algorithmic_bytes(w, S: int, R: int, fusion: bool = True) -> dict:
+def algorithmic_bytes(w, S: int, R: int, fusion: bool = True, kept_rows=None) -> dict:
+    """kept_rows: (layer, batch, recomputed token, KV head) combinations whose head kept the token.  Every listed
+    combination reads its new K and V row; only the kept ones read the old rows (fusion) and write the result.
+    None charges every combination as kept.  The inverse map (4 B per token, memset + scatter) and the scores /
+    index lists are not charged."""
     e = w.elem_bytes
     row = w.head_dim * e
     slabs = w.n_layers * w.batch * w.n_kv_heads
     kbytes = slabs * w.l_tot * row
     score = kbytes                                        # every K row once
     gather = slabs * S * row * 4                          # read K,V rows, write Kc,Vc rows
-    upd = w.n_layers * w.batch * R * w.n_kv_heads * row * (6 if fusion else 4)
+    listed = w.n_layers * w.batch * R * w.n_kv_heads
+    kept = listed if kept_rows is None else int(kept_rows)
+    upd = (2 * listed + (4 if fusion else 2) * kept) * row
     attn = slabs * (S + w.q_tokens) * row * 2             # attention reads Kc,Vc (cache + chunk)
     # decode step i reads the cache as it stands then: S + T_q + i slots (+ its own row)
     dec = sum(slabs * (S + w.q_tokens + i + 1) * row * 2 for i in range(w.decode_steps))
@@ -175,6 +189,7 @@ class Pipeline:
         self.inv_map = torch.empty((L, Bt, Hkv, w.l_tot), dtype=torch.int32, device=device)
         self.O = torch.empty((L, Bt, w.q_tokens, w.n_q_heads, d), dtype=w.torch_dtype, device=device)
         self.R = 0
+        self.update_kept_rows = None
         self.tok_ids = self.Knew = self.Vnew = None
         self.t_loc = self.inp["Qloc"].shape[3]
         self.decode_graph = None
@@ -197,6 +212,11 @@ class Pipeline:
         toks0 = torch.stack([torch.nonzero(inv0[l, 0] >= 0).flatten() for l in range(w.n_layers)])[:, None, :]
         self.R = (w.recompute_share_bp * self.S) // 10000
         self.tok_ids, self.Knew, self.Vnew = synth.make_recompute(w, self.inp["K"], self.inp["V"], toks0, self.R)
+        # rows the update really touches: heads other than head 0 keep only part of the listed tokens
+        kept = 0
+        for l in range(w.n_layers):
+            kept += int((self.inv_map[l][:, :, self.tok_ids[l].long()] >= 0).sum())
+        self.update_kept_rows = kept
 
     def sparsify(self):
         B, inp, w = self.B, self.inp, self.w
@@ -535,6 +555,87 @@ def job_throughput(w, world: int, ms_per_step: float) -> float:
     return w.batch * w.l_tot * world / (ms_per_step / 1e3)
 
 
+def attention_flops(w, S: int) -> float:
+    """QK^T and PV over the visible slots (cache + chunk; the causal part is counted in full), all layers."""
+    return 4.0 * w.n_layers * w.batch * w.q_tokens * w.n_q_heads * (S + w.q_tokens) * w.head_dim
+
+
+def host_description() -> dict:
+    model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except Exception:
+        pass
+    try:
+        allowed = len(os.sched_getaffinity(0))
+    except Exception:
+        allowed = None
+    return {"cpu_model": model, "nproc": os.cpu_count(), "allowed_cpus": allowed}
+
+
+def oracle_one_core_seconds(names=("cfg0", "cfg1")) -> dict:
+    """The oracle's whole path on the small configurations with BLAS limited to one thread."""
+    out = {}
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return out
+    for n in names:
+        w = synth.CONFIGS[n]
+        inp = synth.make_inputs(w, "cpu")
+        with threadpool_limits(limits=1):
+            oracle_sample_seconds(w, inp)
+            out[n] = oracle_sample_seconds(w, inp)
+    return out
+
+
+def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3) -> dict:
+    """Times another configuration with the same code path as the headline one (Pipeline.step: the overlapped
+    schedule where the workload has several layers, in order otherwise), then one in-order pass for the phases."""
+    pipe = Pipeline(w, dev)
+    pipe.prepare_recompute()
+    for _ in range(warmup):
+        pipe.step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        pipe.step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    phase = {}
+    for _ in range(2):
+        ev = []
+        pipe.step(ev, overlap=False)
+        torch.cuda.synchronize()
+        for (n0, a), (n1, b) in zip(ev[:-1], ev[1:]):
+            phase[n1] = phase.get(n1, 0.0) + a.elapsed_time(b) / 2
+    status = max(pipe.B.samkv_poll_status(pipe.handle), pipe.B.samkv_poll_status(pipe.handle_attn))
+    ab = algorithmic_bytes(w, pipe.S, pipe.R, fusion=True, kept_rows=pipe.update_kept_rows)
+    gbs = ab["total"] / (ms / 1e3) / 1e9
+    out = {"layers_or_layer_buffers": w.n_layers, "budget_bp": w.budget_bp, "kept_tokens": pipe.S, "ms_per_step": ms,
+           "us_per_layer": ms * 1e3 / w.n_layers, "algorithmic_gb_per_step": ab["total"] / 1e9, "achieved_gbs": gbs,
+           "frac_of_measured_copy_peak": gbs / hbm_peak, "frac_of_nominal_8tbs": gbs / HBM_NOMINAL_GBS,
+           "schedule": "overlapped (8 layer groups)" if pipe.groups > 1 else "in order",
+           "in_order_phase_ms": phase, "in_order_ms_per_step": sum(phase.values()),
+           "attention_tflops": attention_flops(w, pipe.S) / (phase["attn"] / 1e3) / 1e12 if phase.get("attn") else None,
+           "device_status": status}
+    if w.decode_steps > 0:
+        out["decode"] = {"steps": w.decode_steps, "us_per_step": phase["decode"] * 1e3 / w.decode_steps / w.n_layers,
+                         "achieved_gbs": ab["decode"] / (phase["decode"] / 1e3) / 1e9,
+                         "frac_of_measured_copy_peak": ab["decode"] / (phase["decode"] / 1e3) / 1e9 / hbm_peak,
+                         "frac_of_nominal_8tbs": ab["decode"] / (phase["decode"] / 1e3) / 1e9 / HBM_NOMINAL_GBS,
+                         "launch": "cuda graph"}
+    del pipe
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -547,6 +648,8 @@ def main():
     ap.add_argument("--budget-bp", type=int, default=0, help="override the sequence budget (basis points)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the cfg4 budget sweep, cfg3 and the sustained loop that follow the timed region")
     args = ap.parse_args()
     profiling_case = bool(args.layers or args.batch)       # small captures under a profiler: keep launches few
     if args.warmup < 3 and args.impl == "samkv" and not profiling_case:
@@ -631,12 +734,32 @@ def main():
     sequential_ms = sum(phase_ms.values())
     phase_ms["score"] = timed_phase_ms["score"]          # the roofline figure comes from the timed steps
     widened = widened_rows_ms(pipe) if (rank == 0 and w.decode_steps == 0 and not profiling_case) else None
+    # the same step looped for at least two seconds (board power and clocks settle; the headline region is short)
+    sustained = None
+    if rank == 0 and world == 1 and not profiling_case and not args.no_other_workloads:
+        n_sus = max(20, int(2200.0 / (elapsed_ms / args.steps)))
+        sus_sampler = ClockSampler(local_rank)
+        sus_sampler.start()
+        time.sleep(0.3)
+        torch.cuda.synchronize()
+        sus_sampler.window_open()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(n_sus):
+            pipe.step()
+        s1.record()
+        torch.cuda.synchronize()
+        sus_sampler.window_close()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = s0.elapsed_time(s1) / n_sus
+        sustained = {"steps": n_sus, "ms_per_step": sus_ms, "clocks": sus_clocks,
+                     "mcycles_per_step_at_median_clock": (sus_ms * sus_clocks["sm_mhz"] / 1e3) if sus_clocks.get("sm_mhz") else None}
 
     ms_per_step = elapsed_ms / args.steps
     value = job_throughput(w, world, ms_per_step)
     peaks, peak_kind = measured_peaks()
     hbm_peak = float(peaks.get("hbm_gbs", HBM_FALLBACK_GBS))
-    ab = algorithmic_bytes(w, pipe.S, pipe.R, fusion=True)
+    ab = algorithmic_bytes(w, pipe.S, pipe.R, fusion=True, kept_rows=pipe.update_kept_rows)
     score_gbs = ab["score"] / (phase_ms["score"] / 1e3) / 1e9
     pipeline_gbs = ab["total"] / (ms_per_step / 1e3) / 1e9
 
@@ -655,14 +778,17 @@ def main():
                      "schedule": ("score+select, then %d layer groups: gather+update overlapped with attention on a second stream"
                                   % pipe.groups) if pipe.groups > 1 else "in order on one stream",
                      "timed_phase_ms": timed_phase_ms, "in_order_ms_per_step": sequential_ms,
-                     "phase_ms": phase_ms, "other_calls_ms": widened,
+                     "phase_ms": phase_ms, "other_calls_ms": widened, "sustained": sustained,
+                     "attention_tflops_in_order": attention_flops(w, pipe.S) / (phase_ms["attn"] / 1e3) / 1e12 if phase_ms.get("attn") else None,
+                     "bytes_note": "update charged for the rows it touches (new rows of every listed (token, head), old rows and "
+                                   "results only where the head kept the token); the inverse map and index lists are not charged",
                      "phase_gbs": {k: ab[k] / (phase_ms[k] / 1e3) / 1e9 for k in ("score", "compact", "update", "attn", "decode") if phase_ms.get(k, 0) > 0}},
         "roofline": {"kernel": "score_stream_kernel (with the pooled-query kernel that precedes it in samkv_score)", "bound": "hbm",
                      "achieved": score_gbs, "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": score_gbs / hbm_peak, "frac_of_nominal_8tbs": score_gbs / HBM_NOMINAL_GBS,
                      "algorithmic_bytes_per_launch": ab["score"],
-                     "traffic": (SCORE_KERNEL_DRAM_BYTES_PER_ROW * w.n_layers * w.batch * w.n_kv_heads * w.l_tot
-                                 if (w.dtype == "bf16" and w.head_dim == 128) else None),
+                     "traffic": (score_kernel_dram_bytes_per_row() * w.n_layers * w.batch * w.n_kv_heads * w.l_tot
+                                 if (w.dtype == "bf16" and w.head_dim == 128 and score_kernel_dram_bytes_per_row()) else None),
                      "traffic_note": "ncu dram read+write of a 2-layer launch scaled by rows (profiles/)"},
         "gpu_launches": pipe.launches_per_step() * args.steps,
         "clocks": clocks,
@@ -692,6 +818,27 @@ def main():
                            "note": f"skipped: host has {free / 1e9:.0f} GB free, needs {need / 1e9:.0f} GB pinned"}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, repeats=2)
+        line["cpu_baseline"]["host"] = host_description()
+        if not profiling_case:
+            line["cpu_baseline"]["one_core_seconds_whole_path"] = oracle_one_core_seconds()
+    # the other target configurations, same code path, after the headline one has released its memory
+    if rank == 0 and world == 1 and not profiling_case and not args.no_other_workloads and w.name == "cfg2":
+        del pipe
+        torch.cuda.empty_cache()
+        others = {}
+        ow_sampler = ClockSampler(local_rank)
+        ow_sampler.start()
+        time.sleep(0.3)
+        ow_sampler.window_open()
+        for bp in (500, 1500, 3000, 10000):
+            others[f"cfg4_budget_{bp}bp"] = run_other_workload(synth.CONFIGS["cfg4"].replace(n_layers=32, budget_bp=bp), dev, hbm_peak)
+        others["cfg3"] = run_other_workload(synth.CONFIGS["cfg3"], dev, hbm_peak, steps=5, warmup=2)
+        others["cfg1"] = run_other_workload(synth.CONFIGS["cfg1"], dev, hbm_peak, steps=50, warmup=5)
+        ow_sampler.window_close()
+        others["clocks"] = ow_sampler.stop()
+        others["note"] = ("cfg4: one shape, 32 independent layer buffers, per-layer figures; cfg3: compaction and prefill, then 128 "
+                          "decode steps replayed from one CUDA graph; cfg1: a single small layer (launch-latency bound)")
+        line["pipeline"]["other_workloads"] = others
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
