@@ -253,6 +253,8 @@ class Pipeline:
             side.wait_stream(main)
             for g in range(self.groups):
                 sl = slice(g * per, (g + 1) * per)
+                # (the fused samkv_select_compact is 0.07 ms faster than select + compact on its own, but its larger
+                # CTAs lose more next to the attention kernels than that: 3.49 against 3.38 ms per step)
                 B.samkv_compact(self.handle, shape_g, inp["K"][sl], inp["V"][sl], self.sel[sl], self.k_units, self.Kc[sl],
                                 self.Vc[sl], self.capacity, self.cache_len[sl], self.inv_map[sl])
                 if self.R > 0:

@@ -153,6 +153,23 @@ samkv_status_t samkv_compact(samkv_handle_t h, const samkv_shape_t* shape, const
                              const int32_t* sel, const int32_t* k_units, void* Kc, void* Vc, int32_t cache_capacity,
                              int32_t* cache_len, int32_t* inv_map, void* stream);
 
+/* Selection and compaction in one launch (Sec. 3.2: score -> select -> initial + selected + local rows joined in
+ * their original order).  Same results, bit for bit, as samkv_select followed by samkv_compact: sel_out, Kc, Vc,
+ * cache_len and inv_map are written exactly as those two calls write them; one CTA selects the units of one
+ * (layer, batch, KV head, context) and gathers their rows right away.  Arguments and errors as for the two calls
+ * (V may be pinned host memory). */
+samkv_status_t samkv_select_compact(samkv_handle_t h, const samkv_shape_t* shape, const float* scores,
+                                    const int32_t* k_units, const void* K, const void* V, int32_t* sel_out, void* Kc,
+                                    void* Vc, int32_t cache_capacity, int32_t* cache_len, int32_t* inv_map, void* stream);
+
+/* The whole sparsification in one call: samkv_score, then samkv_select_compact.  scores_out and sel_out are outputs
+ * like those of the separate calls (and must be given: the steps hand their data over through them).  Every argument
+ * is validated before anything is enqueued. */
+samkv_status_t samkv_sparsify(samkv_handle_t h, const samkv_shape_t* shape, const void* K, const void* V, const void* Q,
+                              int32_t T_q, const void* Qloc, int32_t T_loc, int32_t use_bias, const int32_t* k_units,
+                              float* scores_out, int32_t* sel_out, void* Kc, void* Vc, int32_t cache_capacity,
+                              int32_t* cache_len, int32_t* inv_map, void* stream);
+
 /* Composite cache of the protected positions only (Sec. 3.1 "Generate generic query vector": the initial and
  * local K/V of all contexts, concatenated; also the "no-selection" ablation of Sec. 4.1).  Same result as
  * samkv_select with k_units = protected units followed by samkv_compact, without scores or a unit list: the

@@ -27,7 +27,8 @@ EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
            "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
            "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected",
-           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count"]
+           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count", "samkv_select_compact",
+           "samkv_sparsify"]
 
 
 class SamkvError(RuntimeError):
@@ -69,6 +70,8 @@ def lib() -> ctypes.CDLL:
     L.samkv_select.argtypes = [vp, shp, vp, i32p, vp, vp]
     L.samkv_compact.argtypes = [vp, shp, vp, vp, vp, i32p, vp, vp, i32, vp, vp, vp]
     L.samkv_update.argtypes = [vp, shp, vp, vp, i32, vp, vp, i32, vp, vp, i32, vp]
+    L.samkv_select_compact.argtypes = [vp, shp, vp, i32p, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+    L.samkv_sparsify.argtypes = [vp, shp, vp, vp, vp, i32, vp, i32, i32, i32p, vp, vp, vp, vp, i32, vp, vp, vp]
     L.samkv_attn.argtypes = [vp, shp, i32, vp, vp, i32, vp, vp, i32, vp, vp, f32, vp, vp, vp]
     L.samkv_score_static.argtypes = [shp, vp, vp, i32, vp, i32, i32, vp, vp]
     f32p = ctypes.POINTER(ctypes.c_float)
@@ -215,6 +218,20 @@ def samkv_compact(handle: Handle, shape: Shape, K, V, sel, k_units: Sequence[int
     _check(lib().samkv_compact(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(sel),
                                _i32_array(k_units), _ptr(Kc),
                                _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()), "samkv_compact")
+
+
+def samkv_select_compact(handle: Handle, shape: Shape, scores, k_units: Sequence[int], K, V, sel_out, Kc, Vc,
+                         cache_capacity: int, cache_len, inv_map=None):
+    _check(lib().samkv_select_compact(handle.h, shape.ref(), _ptr(scores), _i32_array(k_units), _ptr(K),
+                                      _ptr(V, allow_pinned_host=True), _ptr(sel_out), _ptr(Kc), _ptr(Vc), cache_capacity,
+                                      _ptr(cache_len), _ptr(inv_map), _stream()), "samkv_select_compact")
+
+
+def samkv_sparsify(handle: Handle, shape: Shape, K, V, Q, T_q: int, Qloc, T_loc: int, use_bias: int,
+                   k_units: Sequence[int], scores_out, sel_out, Kc, Vc, cache_capacity: int, cache_len, inv_map=None):
+    _check(lib().samkv_sparsify(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(Q), T_q, _ptr(Qloc),
+                                T_loc, int(use_bias), _i32_array(k_units), _ptr(scores_out), _ptr(sel_out), _ptr(Kc),
+                                _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()), "samkv_sparsify")
 
 
 def samkv_update(handle: Handle, shape: Shape, Kc, Vc, cache_capacity: int, inv_map, tok_ids, R: int, Knew, Vnew,

@@ -294,6 +294,55 @@ samkv_status_t samkv_compact(samkv_handle_t handle, const samkv_shape_t* shape, 
                                   h->d_status, static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_select_compact(samkv_handle_t handle, const samkv_shape_t* shape, const float* scores,
+                                    const int32_t* k_units, const void* K, const void* V, int32_t* sel_out, void* Kc,
+                                    void* Vc, int32_t cache_capacity, int32_t* cache_len, int32_t* inv_map, void* stream) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (scores == nullptr || sel_out == nullptr || K == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr ||
+      cache_len == nullptr)
+    return SAMKV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc)) return SAMKV_ERR_INVALID_ARG;
+  SelTable sel;
+  int S = 0;
+  st = make_sel_table(shape, lo, k_units, &sel, &S);
+  if (st != SAMKV_OK) return st;
+  if (cache_capacity < S) return SAMKV_ERR_CAPACITY;
+  if ((size_t)lo.max_units * 4 + 8192 > (size_t)h->max_smem_optin) return SAMKV_ERR_UNSUPPORTED;
+  return from_cuda(launch_select_compact(*shape, lo.ct, sel, scores, lo.max_units, sel_out, K, V, Kc, Vc, cache_capacity, S,
+                                         cache_len, inv_map, static_cast<cudaStream_t>(stream)));
+}
+
+samkv_status_t samkv_sparsify(samkv_handle_t handle, const samkv_shape_t* shape, const void* K, const void* V,
+                              const void* Q, int32_t T_q, const void* Qloc, int32_t T_loc, int32_t use_bias,
+                              const int32_t* k_units, float* scores_out, int32_t* sel_out, void* Kc, void* Vc,
+                              int32_t cache_capacity, int32_t* cache_len, int32_t* inv_map, void* stream) {
+  // every argument is checked before anything is enqueued: the two calls below validate on the host first, and the
+  // second one's checks are repeated here so that a refusal leaves nothing half done
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  Layout lo;
+  st = make_layout(shape, &lo);
+  if (st != SAMKV_OK) return st;
+  if (sel_out == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || cache_len == nullptr) return SAMKV_ERR_INVALID_ARG;
+  if (!aligned16(V) || !aligned16(Kc) || !aligned16(Vc)) return SAMKV_ERR_INVALID_ARG;
+  SelTable sel;
+  int S = 0;
+  st = make_sel_table(shape, lo, k_units, &sel, &S);
+  if (st != SAMKV_OK) return st;
+  if (cache_capacity < S) return SAMKV_ERR_CAPACITY;
+  if ((size_t)lo.max_units * 4 + 8192 > (size_t)h->max_smem_optin) return SAMKV_ERR_UNSUPPORTED;
+  st = samkv_score(handle, shape, K, Q, T_q, Qloc, T_loc, use_bias, scores_out, nullptr, stream);
+  if (st != SAMKV_OK) return st;
+  return samkv_select_compact(handle, shape, scores_out, k_units, K, V, sel_out, Kc, Vc, cache_capacity, cache_len, inv_map,
+                              stream);
+}
+
 samkv_status_t samkv_compact_protected(samkv_handle_t handle, const samkv_shape_t* shape, const void* K, const void* V,
                                        void* Kc, void* Vc, int32_t cache_capacity, int32_t* cache_len,
                                        int32_t* inv_map, void* stream) {

@@ -42,6 +42,9 @@ cudaError_t launch_score(const samkv_shape_t& s, const CtxTable& ct, const void*
                          int* d_status, cudaStream_t stream);
 cudaError_t launch_select(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const float* scores,
                           const int32_t* k_units_host, int max_units, int32_t* sel, int* d_status, cudaStream_t stream);
+cudaError_t launch_select_compact(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const float* scores,
+                                  int max_units, int32_t* sel, const void* K, const void* V, void* Kc, void* Vc,
+                                  int capacity, int S, int32_t* cache_len, int32_t* inv_map, cudaStream_t stream);
 cudaError_t launch_compact(const samkv_shape_t& s, const CtxTable& ct, const SelTable& st, const void* K, const void* V,
                            const int32_t* sel, void* Kc, void* Vc, int capacity, int S, int32_t* cache_len,
                            int32_t* inv_map, int* d_status, cudaStream_t stream);

@@ -365,6 +365,77 @@ def test_chunked_prefill_on_the_tensor_memory_kernel():
         assert np.array_equal(to_f64(run.Kc[0, b])[:, :n], Kc_ref[b][:, :n])
 
 
+@pytest.mark.parametrize("case", ["cfg0", "cfg1", "ragged_f32", "ragged_bf16_d64", "blocks16", "paper_blocks", "all_kept",
+                                  "protected_only"])
+def test_sparsify_in_one_call_equals_the_three_calls(case):
+    """samkv_sparsify (score, then selection and gather fused in one launch) and samkv_select_compact write exactly
+    what samkv_score + samkv_select + samkv_compact write: scores, unit list, compact cache, cache length and inverse
+    map, bit for bit."""
+    k_units = None
+    if case in ("cfg0", "cfg1"):
+        w = synth.CONFIGS[case]
+    elif case == "ragged_f32":
+        w = synth.ragged_workload(dtype="f32", head_dim=64)
+    elif case == "ragged_bf16_d64":
+        w = synth.ragged_workload(dtype="bf16", head_dim=64, n_q_heads=8, n_kv_heads=2)
+    elif case == "blocks16":
+        w = synth.ragged_workload(ctx_lens=(160, 257, 64, 1000), dtype="bf16", head_dim=128, block_size=16, n_init=16, n_local=32)
+    elif case == "paper_blocks":
+        w = synth.CONFIGS["cfg1"].replace(block_size=64, n_init=64, n_local=128)
+    else:
+        w = synth.ragged_workload(dtype="bf16", head_dim=128)
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    shape = B.Shape.from_workload(w)
+    if case == "all_kept":
+        prot, U_tot, _ = B.samkv_layout(shape)
+        k_units = [-(-n // w.block_size) for n in w.ctx_lens]
+    elif case == "protected_only":
+        k_units = list(B.samkv_layout(shape)[0])
+    ref = DeviceRun(w, inp, k_units=k_units).sparsify()
+    torch.cuda.synchronize()
+    for fused_score in (True, False):
+        got = DeviceRun(w, inp, k_units=k_units)
+        got.Kc.fill_(7.0); got.Vc.fill_(7.0); got.inv_map.fill_(123)
+        ref2 = DeviceRun(w, inp, k_units=k_units)
+        ref2.Kc.fill_(7.0); ref2.Vc.fill_(7.0); ref2.inv_map.fill_(123)
+        ref2.sparsify()
+        if fused_score:
+            B.samkv_sparsify(got.handle, got.shape, inp["K"], inp["V"], inp["Q"], w.q_tokens, inp["Qloc"],
+                             inp["Qloc"].shape[3], 1, got.k_units, got.scores, got.sel, got.Kc, got.Vc, got.capacity,
+                             got.cache_len, got.inv_map)
+        else:
+            B.samkv_select_compact(got.handle, got.shape, ref.scores, got.k_units, inp["K"], inp["V"], got.sel, got.Kc,
+                                   got.Vc, got.capacity, got.cache_len, got.inv_map)
+        torch.cuda.synchronize()
+        assert got.poll() == 0
+        if fused_score:
+            assert torch.equal(got.scores, ref2.scores)
+        assert torch.equal(got.sel, ref2.sel)
+        assert torch.equal(got.cache_len, ref2.cache_len)
+        assert torch.equal(got.inv_map, ref2.inv_map)
+        view = torch.int16 if w.dtype == "bf16" else torch.int32
+        assert torch.equal(got.Kc.view(view), ref2.Kc.view(view))       # untouched tail slots included
+        assert torch.equal(got.Vc.view(view), ref2.Vc.view(view))
+
+
+def test_sparsify_refuses_bad_arguments_before_launching_anything():
+    w = synth.CONFIGS["cfg0"]
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = DeviceRun(w, inp)
+    run.scores.fill_(-3.0)
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_sparsify(run.handle, run.shape, inp["K"], inp["V"], inp["Q"], w.q_tokens, inp["Qloc"], inp["Qloc"].shape[3],
+                         1, run.k_units, run.scores, run.sel, run.Kc, run.Vc, run.S - 1, run.cache_len, run.inv_map)
+    assert e.value.status == 4                                            # capacity
+    with pytest.raises(B.SamkvError) as e:
+        B.samkv_sparsify(run.handle, run.shape, inp["K"], inp["V"], inp["Q"], w.q_tokens, inp["Qloc"], inp["Qloc"].shape[3],
+                         1, [10 ** 6] * w.n_ctx, run.scores, run.sel, run.Kc, run.Vc, run.capacity, run.cache_len,
+                         run.inv_map)
+    assert e.value.status == 5                                            # budget
+    torch.cuda.synchronize()
+    assert bool((run.scores == -3.0).all())                               # the scoring step was not enqueued either
+
+
 def test_attention_sees_q_written_by_the_kernel_right_before_it():
     """Stream order on Q: a kernel on the same stream writes Q immediately before every one of several hundred
     back-to-back attention calls on the tensor-memory path (which is launched as a programmatic dependent and
