@@ -48,12 +48,23 @@ class samkv_shape_t(ctypes.Structure):
 def lib() -> ctypes.CDLL:
     """Loads libsamkv.so (built by `python -m paper_2508_11661_b200.build`).  Raises if it is missing."""
     global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(_LIB_PATH):
-        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2508_11661_b200.build` "
+    if _lib is None:
+        _lib = load_library(_LIB_PATH)
+    return _lib
+
+
+def use_library(path: str) -> None:
+    """Makes every function of this module call the library at `path` from now on (the tests of the debug build load
+    libsamkv_debug.so this way); handles created before the switch must not be used after it."""
+    global _lib
+    _lib = load_library(path)
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2508_11661_b200.build` "
                            "(the SamKV CUDA library has no CPU fallback)")
-    L = ctypes.CDLL(_LIB_PATH)
+    L = ctypes.CDLL(path)
     vp, i32, sz, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t, ctypes.c_float
     shp = ctypes.POINTER(samkv_shape_t)
     i32p = ctypes.POINTER(ctypes.c_int32)
@@ -90,7 +101,8 @@ def lib() -> ctypes.CDLL:
     for name in EXPORTS:
         if name not in ("samkv_status_string", "samkv_workspace_bytes", "samkv_select_cross_scratch_bytes"):
             getattr(L, name).restype = ctypes.c_int
-    _lib = L
+    if hasattr(L, "samkv_debug_score_with_lost_copy"):          # only the debug build exports it
+        L.samkv_debug_score_with_lost_copy.argtypes = [vp, shp, vp, vp, i32, vp, i32, i32, vp, ctypes.c_uint32, vp]
     return L
 
 

@@ -10,6 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsamkv.so")
+DEBUG_LIB_PATH = os.path.join(PKG_DIR, "libsamkv_debug.so")   # same sources with -DSAMKV_DEBUG_CHECKS (test hooks)
 SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "topp.cu", "align.cu", "means.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu", "attn_tc4.cu"]
 
 
@@ -20,22 +21,26 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _stale(lib_path: str = LIB_PATH) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(lib_path)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "samkv.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB_PATH
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """debug=True builds libsamkv_debug.so: the same library plus the hooks a test needs to make a bounded wait run out."""
+    lib_path = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not force and not _stale(lib_path):
+        return lib_path
     objs = []
-    build_dir = os.path.join(PKG_DIR, "build")
+    build_dir = os.path.join(PKG_DIR, "build", "debug" if debug else "release")
     os.makedirs(build_dir, exist_ok=True)
     common = [nvcc_path(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    if debug:
+        common += ["-DSAMKV_DEBUG_CHECKS"]
     if verbose:
         common += ["-Xptxas", "-v"]
     procs = []
@@ -50,9 +55,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}")
-    subprocess.check_call([nvcc_path(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs)
-    return LIB_PATH
+    subprocess.check_call([nvcc_path(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib_path] + objs)
+    return lib_path
 
 
 if __name__ == "__main__":
     print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, debug=True))

@@ -5,6 +5,8 @@
 
 #include <new>
 
+#include <stdio.h>
+
 #include "common.cuh"
 
 using namespace samkv;
@@ -110,7 +112,12 @@ samkv_status_t check_handle(samkv_ctx_impl* h) {
   return SAMKV_OK;
 }
 
-inline samkv_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? SAMKV_OK : SAMKV_ERR_CUDA; }
+inline samkv_status_t from_cuda(cudaError_t e) {
+#ifdef SAMKV_DEBUG_CHECKS
+  if (e != cudaSuccess) fprintf(stderr, "samkv (debug build): CUDA error %d: %s\n", (int)e, cudaGetErrorString(e));
+#endif
+  return e == cudaSuccess ? SAMKV_OK : SAMKV_ERR_CUDA;
+}
 
 }  // namespace
 
@@ -251,7 +258,7 @@ samkv_status_t samkv_score(samkv_handle_t handle, const samkv_shape_t* shape, co
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = launch_qhat(*shape, Q, T_q, Qloc, T_loc, use_bias, qhat, s);
-  if (e != cudaSuccess) return SAMKV_ERR_CUDA;
+  if (e != cudaSuccess) return from_cuda(e);
   return from_cuda(launch_score(*shape, lo.ct, K, qhat, scores_out, h->d_status, s));
 }
 
@@ -378,7 +385,7 @@ samkv_status_t samkv_update(samkv_handle_t handle, const samkv_shape_t* shape, v
   if (Kc == nullptr || Vc == nullptr || inv_map == nullptr || tok_ids == nullptr || Knew == nullptr || Vnew == nullptr)
     return SAMKV_ERR_INVALID_ARG;
   if (!aligned16(Kc) || !aligned16(Vc) || !aligned16(Knew) || !aligned16(Vnew)) return SAMKV_ERR_INVALID_ARG;
-  return from_cuda(launch_update(*shape, lo.L_tot, Kc, Vc, cache_capacity, inv_map, tok_ids, R, Knew, Vnew, mode,
+  return from_cuda(launch_update(*shape, lo.L_tot, Kc, Vc, cache_capacity, inv_map, tok_ids, R, Knew, Vnew, mode, h->d_status,
                                  static_cast<cudaStream_t>(stream)));
 }
 
@@ -574,3 +581,24 @@ samkv_status_t samkv_align(samkv_handle_t handle, const samkv_shape_t* shape, co
 }
 
 }  // extern "C"
+
+#ifdef SAMKV_DEBUG_CHECKS
+namespace samkv {
+cudaError_t debug_set_score_wait(uint32_t spin_limit, int withhold_first_tile, cudaStream_t stream);
+}
+// Debug build only (libsamkv_debug.so): samkv_score with the scoring kernel's waits shortened to `spin_limit` polls and
+// the copies of every CTA's first tile withheld, so that the bounded wait for that tile runs out.  The kernel records
+// the device check, drains and returns; samkv_poll_status then reports SAMKV_ERR_DEVICE_CHECK and later calls work as
+// usual.  scores_out is left partly unwritten.
+extern "C" samkv_status_t samkv_debug_score_with_lost_copy(samkv_handle_t handle, const samkv_shape_t* shape, const void* K,
+                                                           const void* Q, int32_t T_q, const void* Qloc, int32_t T_loc,
+                                                           int32_t use_bias, float* scores_out, uint32_t spin_limit,
+                                                           void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (samkv::debug_set_score_wait(spin_limit, 1, s) != cudaSuccess) return SAMKV_ERR_CUDA;
+  const samkv_status_t st = samkv_score(handle, shape, K, Q, T_q, Qloc, T_loc, use_bias, scores_out, nullptr, stream);
+  if (samkv::debug_set_score_wait(0, 0, s) != cudaSuccess) return SAMKV_ERR_CUDA;
+  return st;
+}
+#endif
+

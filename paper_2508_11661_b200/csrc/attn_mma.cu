@@ -275,7 +275,7 @@ static cudaError_t launch_mma_t(const samkv_shape_t& s, const void* Kc, const vo
   const int smem = kBM * kHeadDim * 2 + 4 * kBN * kHeadDim * 2;
   auto kern = attn_mma_kernel<kHeadDim, kWarps>;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = ensure_dynamic_smem<2000 + kHeadDim * 16 + kWarps>(kern, smem);
     if (e != cudaSuccess) return e;
   }
   kern<<<(unsigned)blocks, kWarps * 32, smem, stream>>>(

@@ -381,7 +381,7 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
   if (!tc::make_kv_map(&tmK, Kc, capacity, s.batch * s.n_kv_heads) ||
       !tc::make_kv_map(&tmV, Vc, capacity, s.batch * s.n_kv_heads))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::kSmemBytes);
+  cudaError_t e = ensure_dynamic_smem<3>(attn_tc2_kernel, tc2::kSmemBytes);
   if (e != cudaSuccess) return e;
   // Launched so that it may start while the kernel before it in the stream (the append of the chunk) is still
   // running: set-up and the Q loads need nothing from it; the loader waits before its first K/V tile.

@@ -627,7 +627,7 @@ cudaError_t launch_attn_tc4(const samkv_shape_t& s, void* Kc, void* Vc, int capa
     return cudaErrorInvalidValue;
   const bool pair = attn_merges_in_cluster(plan);
   auto kern = pair ? attn_tc4_kernel<true> : attn_tc4_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc4::kSmemBytes);
+  cudaError_t e = pair ? ensure_dynamic_smem<1>(kern, tc4::kSmemBytes) : ensure_dynamic_smem<2>(kern, tc4::kSmemBytes);
   if (e != cudaSuccess) return e;
   // Launched so that it may start while the kernel before it in the stream is still running: barrier set-up and the
   // tensor-memory allocation need nothing from it; one wait precedes every read.

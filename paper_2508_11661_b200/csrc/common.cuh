@@ -49,7 +49,7 @@ cudaError_t launch_compact(const samkv_shape_t& s, const CtxTable& ct, const Sel
                            const int32_t* sel, void* Kc, void* Vc, int capacity, int S, int32_t* cache_len,
                            int32_t* inv_map, int* d_status, cudaStream_t stream);
 cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc, int capacity, const int32_t* inv_map,
-                          const int32_t* tok_ids, int R, const void* Knew, const void* Vnew, int mode,
+                          const int32_t* tok_ids, int R, const void* Knew, const void* Vnew, int mode, int* d_status,
                           cudaStream_t stream);
 
 cudaError_t launch_topp(const samkv_shape_t& s, const CtxTable& ct, const int* n_init_units, const int* first_local_unit,
@@ -85,10 +85,28 @@ cudaError_t launch_attn(const samkv_shape_t& s, int layer, void* Kc, void* Vc, i
                         const void* Q, int T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
                         void* partial_ws, const AttnPlan& plan, int* d_status, cudaStream_t stream);
 
+// Raises a kernel's dynamic shared-memory limit to `bytes`; the runtime call is made only when this process has not
+// yet set at least that much for this kernel on the current device (the setting is per device and sticks), so that
+// repeated calls of an entry point cost nothing.  One static slot per instantiation (kTag distinguishes call sites).
+// Internal linkage on purpose: with external linkage the slot would be shared between two copies of this library
+// loaded into one process (the regular and the debug build), and the second copy would skip its own kernels.
+template <int kTag, typename Kernel>
+static cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes) {
+  constexpr int kMaxDev = 64;
+  static int granted[kMaxDev] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < kMaxDev && granted[dev] >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && dev >= 0 && dev < kMaxDev) granted[dev] = bytes;
+  return e;
+}
+
 // ----- small device helpers ---------------------------------------------------------------------------
 enum DeviceCheck : int {
   CHECK_OK = 0,
-  CHECK_SEL_RANGE = 1,      // a selected unit id lies outside its context
+  CHECK_SEL_RANGE = 1,      // a selected unit id lies outside its context, or a recomputed token / its slot is out of range
   CHECK_APPEND_CAPACITY = 2, // cache_len + T_q exceeds the cache capacity
   CHECK_WAIT_TIMEOUT = 3,    // a bounded wait on an mbarrier ran out
   CHECK_SMEM_ALIGNMENT = 4,  // dynamic shared memory not aligned as the tensor-core tiles need

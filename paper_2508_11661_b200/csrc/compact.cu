@@ -133,7 +133,7 @@ template <typename T, int kHeadDim>
 __global__ void __launch_bounds__(kCopyThreads)
 update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict__ inv_map,
               const int32_t* __restrict__ tok_ids, const T* __restrict__ Knew, const T* __restrict__ Vnew, int Bt,
-              int Hkv, int R, int L_tot, int capacity, int mode, long long n_rows) {
+              int Hkv, int R, int L_tot, int capacity, int mode, long long n_rows, int* __restrict__ d_status) {
   constexpr int kPerVec = ElemTraits<T>::kPerVec;
   constexpr int kLanes = kHeadDim / kPerVec;
   constexpr int kRowsPerCta = kCopyThreads / kLanes;
@@ -160,7 +160,11 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
     const int t = tok_ids[(size_t)l * R + r];
     slab = (size_t)lb * Hkv + h;
     if (t >= 0 && t < L_tot) slot = inv_map[slab * L_tot + t];
-    if (slot >= capacity) slot = -1;
+    // a token id past the sequence or a slot past the cache is skipped and reported (-1 is the regular "skip")
+    if (t >= L_tot || t < -1 || slot >= capacity) {
+      if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);
+      slot = -1;
+    }
   }
   active = slot >= 0;
   size_t dst = 0;
@@ -182,7 +186,7 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
 }
 
 cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc, int capacity, const int32_t* inv_map,
-                          const int32_t* tok_ids, int R, const void* Knew, const void* Vnew, int mode,
+                          const int32_t* tok_ids, int R, const void* Knew, const void* Vnew, int mode, int* d_status,
                           cudaStream_t stream) {
   const long long n_rows = (long long)s.n_layers * s.batch * R * s.n_kv_heads;
   if (n_rows == 0) return cudaSuccess;
@@ -195,7 +199,7 @@ cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc,
     update_kernel<T, HD><<<dim3((unsigned)per_lb, (unsigned)n_lb), kCopyThreads, 0, stream>>>((T*)Kc, (T*)Vc, inv_map, tok_ids, \
                                                                        (const T*)Knew, (const T*)Vnew, s.batch,    \
                                                                        s.n_kv_heads, R, L_tot, capacity, mode,     \
-                                                                       n_rows);                                    \
+                                                                       n_rows, d_status);                          \
   } while (0)
   if (s.dtype == SAMKV_BF16) {
     if (s.head_dim == 128) SAMKV_LAUNCH_UPDATE(__nv_bfloat16, 128); else SAMKV_LAUNCH_UPDATE(__nv_bfloat16, 64);

@@ -247,8 +247,18 @@ struct TileTable {
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+#ifdef SAMKV_DEBUG_CHECKS
+// Debug build only: a test can shorten the wait limit and make the producer withhold the copies of its first tile,
+// so that the consumers' wait for that tile runs out.  Nothing faults or hangs: every wait stays bounded.
+__device__ uint32_t g_debug_spin_limit = 0;     // 0 = the regular limit
+__device__ int g_debug_withhold_first_tile = 0;
+#define SAMKV_SCORE_SPIN_LIMIT (g_debug_spin_limit ? g_debug_spin_limit : kScoreSpinLimit)
+#else
+#define SAMKV_SCORE_SPIN_LIMIT kScoreSpinLimit
+#endif
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kScoreSpinLimit; ++i) {
+  const uint32_t limit = SAMKV_SCORE_SPIN_LIMIT;
+  for (uint32_t i = 0; i < limit; ++i) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -321,6 +331,9 @@ score_stream_kernel(const T* __restrict__ K, const float* __restrict__ qhat, flo
         const T* src = K + (slab * L_tot + ct.ctx_off[c] + row0) * kHeadDim;
         const float* qsrc = qhat + (((slab / Hkv) * ct.n_ctx + c) * Hkv + slab % Hkv) * kHeadDim;
         const uint32_t bar = full0 + 8 * stage;
+#ifdef SAMKV_DEBUG_CHECKS
+        if (g_debug_withhold_first_tile && n == 0) continue;      // the consumers' wait for this tile runs out
+#endif
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes + kQBytes) : "memory");
         asm volatile(
             "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
@@ -430,7 +443,7 @@ static cudaError_t launch_score_t(const samkv_shape_t& s, const CtxTable& ct, co
   const size_t smem = (size_t)kStages * (kTileBytesMax + kHeadDim * sizeof(float) + kRows * sizeof(float) + 16) +
                       2 * kStages * 8 + 16;
   auto kern = score_stream_kernel<T, kHeadDim>;
-  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  e = ensure_dynamic_smem<100 + kHeadDim>(kern, (int)smem);
   if (e != cudaSuccess) return e;
   const long long grid = total_tiles < 2LL * sms ? total_tiles : 2LL * sms;
   kern<<<(unsigned)grid, kStreamThreads, smem, stream>>>((const T*)K, qhat, scores, ct, tt, s.n_kv_heads,
@@ -448,5 +461,14 @@ cudaError_t launch_score(const samkv_shape_t& s, const CtxTable& ct, const void*
   if (s.head_dim == 128) return launch_score_t<float, 128>(s, ct, K, qhat, scores, d_status, stream);
   return launch_score_t<float, 64>(s, ct, K, qhat, scores, d_status, stream);
 }
+
+#ifdef SAMKV_DEBUG_CHECKS
+cudaError_t debug_set_score_wait(uint32_t spin_limit, int withhold_first_tile, cudaStream_t stream) {
+  cudaError_t e = cudaMemcpyToSymbolAsync(g_debug_spin_limit, &spin_limit, sizeof(spin_limit), 0, cudaMemcpyHostToDevice, stream);
+  if (e != cudaSuccess) return e;
+  return cudaMemcpyToSymbolAsync(g_debug_withhold_first_tile, &withhold_first_tile, sizeof(int), 0, cudaMemcpyHostToDevice,
+                                 stream);
+}
+#endif
 
 }  // namespace samkv

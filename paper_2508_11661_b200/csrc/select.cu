@@ -210,7 +210,7 @@ cudaError_t launch_select(const samkv_shape_t& s, const CtxTable& ct, const SelT
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)max_units * sizeof(uint32_t);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem<6>(select_kernel, (int)smem);
     if (e != cudaSuccess) return e;
   }
   (void)d_status;
@@ -229,8 +229,7 @@ static cudaError_t launch_select_compact_t(const samkv_shape_t& s, const CtxTabl
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   const size_t smem = (size_t)max_units * sizeof(uint32_t);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(select_compact_kernel<kRowBytes>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = ensure_dynamic_smem<1000 + kRowBytes>(select_compact_kernel<kRowBytes>, (int)smem);
     if (e != cudaSuccess) return e;
   }
   const int L_tot = ct.ctx_off[ct.n_ctx];

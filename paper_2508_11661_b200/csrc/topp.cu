@@ -436,7 +436,7 @@ cudaError_t launch_select_cross(const samkv_shape_t& s, const CtxTable& ct, cons
     const size_t smem = (size_t)n_mid_max * sizeof(uint32_t);
     if (smem + 2048 > (size_t)max_smem_optin) return cudaErrorInvalidConfiguration;
     if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(retrieve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      cudaError_t e = ensure_dynamic_smem<8>(retrieve_kernel, (int)smem);
       if (e != cudaSuccess) return e;
     }
     retrieve_kernel<<<(unsigned)(slabs * ct.n_ctx), kRetrieveThreads, smem, stream>>>(scores, ckey, cid, ct, tt, U_tot, C_tot);

@@ -10,6 +10,9 @@ from paper_2508_11661_b200 import binding as B
 from paper_2508_11661_b200 import synth
 
 
+CANARY, CANARY_WORDS = 12345, 64
+
+
 def to_f64(t: torch.Tensor) -> np.ndarray:
     """Exact up-conversion of stored bf16 / fp32 values."""
     return t.detach().to("cpu").to(torch.float64).numpy()
@@ -33,9 +36,23 @@ class DeviceRun:
         dev = inp["K"].device
         L, Bt, Hkv, d = w.n_layers, w.batch, w.n_kv_heads, w.head_dim
         self.handle = B.Handle(self.shape, max(w.q_tokens, 1), self.capacity)
-        self.scores = torch.empty((L, Bt, Hkv, self.U_tot), dtype=torch.float32, device=dev)
-        self.qhat = torch.empty((L, Bt, w.n_ctx, Hkv, d), dtype=torch.float32, device=dev)
-        self.sel = torch.full((L, Bt, Hkv, sum(self.k_units)), -7, dtype=torch.int32, device=dev)
+        # outputs sit in front of canary words that no kernel may touch (checked by poll())
+        self._guarded = []
+
+        def guarded(shape, dtype, fill=None):
+            n = 1
+            for v in shape:
+                n *= v
+            flat = torch.empty(n + CANARY_WORDS, dtype=dtype, device=dev)
+            flat[n:] = CANARY
+            if fill is not None:
+                flat[:n] = fill
+            self._guarded.append(flat[n:])
+            return flat[:n].view(shape)
+
+        self.scores = guarded((L, Bt, Hkv, self.U_tot), torch.float32)
+        self.qhat = guarded((L, Bt, w.n_ctx, Hkv, d), torch.float32)
+        self.sel = guarded((L, Bt, Hkv, sum(self.k_units)), torch.int32, fill=-7)
         self.Kc = torch.zeros((L, Bt, Hkv, self.capacity, d), dtype=w.torch_dtype, device=dev)
         self.Vc = torch.zeros_like(self.Kc)
         self.cache_len = torch.zeros((L, Bt), dtype=torch.int32, device=dev)
@@ -67,7 +84,10 @@ class DeviceRun:
         return Oo, lse
 
     def poll(self):
-        return B.samkv_poll_status(self.handle)
+        status = B.samkv_poll_status(self.handle)        # synchronises the stream
+        for tail in self._guarded:
+            assert bool((tail == CANARY).all()), "a kernel wrote past the end of an output"
+        return status
 
 
 def oracle_scores(w, inp, l, b, use_bias=True, with_qloc=True):
