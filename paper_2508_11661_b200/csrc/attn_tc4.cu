@@ -183,6 +183,7 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   // Everything above needs nothing from the kernels before this one in the stream (they may still be running when
   // this kernel was launched as a programmatic dependent); everything below does: Q, cache_len, the cache rows.
   pdl_wait();
+  int len = cache_len[b];     // (issued first: its latency overlaps the Q copies below)
 
   // Q tile: cp.async by the softmax warps (rows beyond the chunk zero-filled)
   if (warp < kSoftmaxWarps) {
@@ -196,7 +197,6 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
-  int len = cache_len[b];
   len = max(0, min(len, capacity));
   const int n_app = (appended && len + T_q <= capacity) ? T_q : 0;
   const int total = len + n_app;
@@ -215,6 +215,11 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   if (appended && n_app == 0 && blockIdx.x == 0 && tid == 0) atomicMax(d_status, (int)CHECK_APPEND_CAPACITY);
 
   if (warp < kSoftmaxWarps) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(Q_READY));
+    // (after Q has been handed over: the first products do not wait for this copy, only the last tiles do)
     if (copies_chunk) {
       for (int i0 = 0; i0 < T_q * 16; i0 += kSoftmaxWarps * 32 * 4) {      // four rows' pieces in flight per thread
         uint4 vk[4], vv[4];
@@ -241,10 +246,6 @@ attn_tc4_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(APPENDED));
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    fence_proxy_async();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar(Q_READY));
   }
 
   // Waits are executed by every lane of the waiting warp (the warp stays converged; a lone polling lane with the
