@@ -139,10 +139,12 @@ samkv_status_t samkv_select(samkv_handle_t h, const samkv_shape_t* shape, const 
 
 /* Compaction (Sec. 3.2: initial + selected + local rows joined in their original order).
  *   Kc[l,b,h,slot,:] = K[l,b,h,tok(slot),:], same for V; slots run over (context, token) ascending.
- *   K, V      [L, Bt, Hkv, L_tot, d].  V (only V) may also be a pointer into PINNED HOST memory that the
+ *   K, V      [L, Bt, Hkv, L_tot, d].  Either may also be a pointer into PINNED HOST memory that the
  *             device can address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel
- *             then pulls just the kept V rows across the bus, so only the kept share of V is ever loaded
- *             to the GPU (the paper's "sequence ratio", Table 1); K is read on the device by samkv_score anyway
+ *             then pulls just the kept rows across the bus, so only the kept share is ever loaded to the GPU
+ *             (the paper's "sequence ratio", Table 1).  V can always stay on the host; K can when the scores
+ *             came from the block representatives (samkv_score_blocks), since token-mode samkv_score reads
+ *             all of K on the device anyway
  *   sel       int32 [L, Bt, Hkv, S_u] as written by samkv_select; k_units host [n_ctx]
  *   Kc, Vc    [L, Bt, Hkv, cache_capacity, d]; slots >= S are left untouched
  *   cache_len int32 [L, Bt], set to S (the number of kept tokens)
@@ -157,7 +159,7 @@ samkv_status_t samkv_compact(samkv_handle_t h, const samkv_shape_t* shape, const
  * their original order).  Same results, bit for bit, as samkv_select followed by samkv_compact: sel_out, Kc, Vc,
  * cache_len and inv_map are written exactly as those two calls write them; one CTA selects the units of one
  * (layer, batch, KV head, context) and gathers their rows right away.  Arguments and errors as for the two calls
- * (V may be pinned host memory). */
+ * (K and V may be pinned host memory). */
 samkv_status_t samkv_select_compact(samkv_handle_t h, const samkv_shape_t* shape, const float* scores,
                                     const int32_t* k_units, const void* K, const void* V, int32_t* sel_out, void* Kc,
                                     void* Vc, int32_t cache_capacity, int32_t* cache_len, int32_t* inv_map, void* stream);

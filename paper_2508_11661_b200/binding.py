@@ -226,8 +226,8 @@ def samkv_select(handle: Handle, shape: Shape, scores, k_units: Sequence[int], s
 
 def samkv_compact(handle: Handle, shape: Shape, K, V, sel, k_units: Sequence[int], Kc, Vc, cache_capacity: int,
                   cache_len, inv_map=None):
-    # V may live in pinned host memory: the gather then reads only the kept rows across the bus
-    _check(lib().samkv_compact(handle.h, shape.ref(), _ptr(K), _ptr(V, allow_pinned_host=True), _ptr(sel),
+    # K and V may live in pinned host memory: the gather then reads only the kept rows across the bus
+    _check(lib().samkv_compact(handle.h, shape.ref(), _ptr(K, allow_pinned_host=True), _ptr(V, allow_pinned_host=True), _ptr(sel),
                                _i32_array(k_units), _ptr(Kc),
                                _ptr(Vc), cache_capacity, _ptr(cache_len), _ptr(inv_map), _stream()), "samkv_compact")
 

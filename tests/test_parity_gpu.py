@@ -255,8 +255,8 @@ def test_append_past_capacity_is_reported_not_fatal():
     assert torch.equal(Og, Og2)
 
 
-def test_compact_gathers_v_rows_from_pinned_host_memory():
-    """V may stay in pinned host memory; only the kept rows cross the bus.  Same bits as with V on the device."""
+def test_compact_gathers_rows_from_pinned_host_memory():
+    """V (and K) may stay in pinned host memory; only the kept rows cross the bus.  Same bits as from the device."""
     w = synth.CONFIGS["cfg1"]
     inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
     run = DeviceRun(w, inp).sparsify()
@@ -269,6 +269,13 @@ def test_compact_gathers_v_rows_from_pinned_host_memory():
     torch.cuda.synchronize()
     assert torch.equal(run.Kc, Kc_dev) and torch.equal(run.Vc, Vc_dev)
     check_compact(w, run, 0, 0, run.sel[0, 0].cpu().numpy())
+    # K too (the deployment with block representatives resident: neither K nor V is uploaded as a whole)
+    K_host = inp["K"].cpu().pin_memory()
+    run.Kc.zero_(); run.Vc.zero_()
+    B.samkv_compact(run.handle, run.shape, K_host, V_host, run.sel, run.k_units, run.Kc, run.Vc, run.capacity,
+                    run.cache_len, run.inv_map)
+    torch.cuda.synchronize()
+    assert torch.equal(run.Kc, Kc_dev) and torch.equal(run.Vc, Vc_dev)
     with pytest.raises(ValueError):                                   # pageable host memory is refused by the binding
         B.samkv_compact(run.handle, run.shape, inp["K"], inp["V"].cpu(), run.sel, run.k_units, run.Kc, run.Vc,
                         run.capacity, run.cache_len, run.inv_map)
@@ -286,6 +293,19 @@ def test_many_contexts_and_raw_local_query_rows():
     with pytest.raises(B.SamkvError) as e:                              # 129 contexts: refused, not truncated
         B.samkv_budget_units(shape, 1500)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("dtype,hd,lo,hi,n", [("bf16", 128, 24, 25, 20), ("f32", 64, 16, 41, 30), ("f32", 128, 3, 11, 40),
+                                              ("bf16", 64, 33, 71, 25), ("bf16", 128, 100, 400, 7)])
+def test_short_contexts_share_scoring_tiles(dtype, hd, lo, hi, n):
+    """Contexts much shorter than a 32 KB scoring tile: a tile then spans several contexts and every row is scored
+    with the personalised query of its own context (Eq. 1).  The third case has more contexts per tile than the
+    kernel carries queries for (it falls back to one tile per context), the last one mixes both regimes."""
+    g = torch.Generator().manual_seed(hd + n)
+    lens = tuple(int(x) for x in torch.randint(lo, hi, (n,), generator=g))
+    w = synth.Workload("short_ctx", 2, 2, 8, 2, hd, dtype, lens, 6, budget_bp=3000, block_size=1, n_init=1, n_local=2,
+                       t_loc=2, rope_base=10000.0, seed=5)
+    full_check(w)
 
 
 def test_large_context_uses_block_wide_select_and_head_dim_64_prefill():
