@@ -39,6 +39,18 @@ def test_library_exports_every_declared_entry_point():
     assert names == set(B.EXPORTS), "binding.EXPORTS and the header disagree"
 
 
+def test_debug_entry_point_exists_only_in_the_debug_build():
+    """The hook that makes a bounded wait run out is compiled into libsamkv_debug.so alone."""
+    from paper_2508_11661_b200 import build
+    assert not hasattr(B.lib(), "samkv_debug_score_with_lost_copy")
+    if not os.path.exists(build.DEBUG_LIB_PATH):
+        pytest.skip("debug library not built")
+    dbg = B.load_library(build.DEBUG_LIB_PATH)
+    assert hasattr(dbg, "samkv_debug_score_with_lost_copy")
+    for n in declared_symbols():
+        assert hasattr(dbg, n), f"{n} missing from the debug build"
+
+
 def test_status_strings():
     lib = B.lib()
     seen = {lib.samkv_status_string(i).decode() for i in range(8)}
