@@ -980,7 +980,7 @@ def main():
                      "algorithmic_bytes_per_launch": ab["score"],
                      "traffic": (score_kernel_dram_bytes_per_row() * w.n_layers * w.batch * w.n_kv_heads * w.l_tot
                                  if (w.dtype == "bf16" and w.head_dim == 128 and score_kernel_dram_bytes_per_row()) else None),
-                     "traffic_note": "ncu dram read+write of a 2-layer launch scaled by rows (profiles/)"},
+                     "traffic_note": "ncu dram read+write of an 8-layer launch scaled by rows (profiles/)"},
         "gpu_launches": pipe.launches_per_step() * args.steps,
         "clocks": clocks,
     }
