@@ -160,6 +160,9 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # the GPU arm
 # --------------------------------------------------------------------------------------------------
+ATTN_SHARE_SM = "auto"      # --attn-share-sm auto|on|off: which prefill attention kernel the overlapped schedule uses
+
+
 class Pipeline:
     """Device-resident state of one request batch and the calls of one step."""
 
@@ -179,6 +182,11 @@ class Pipeline:
         # that the tensor-bound attention of one layer group overlaps the HBM-bound gather of the next
         self.shape1 = B.Shape.from_workload(w, n_layers=1)
         self.handle_attn = B.Handle(self.shape1, w.q_tokens, self.capacity)
+        # Its kernels run next to the gather and update of the following layers.  samkv_attn_share_sm asks for the
+        # attention kernel that leaves registers and shared memory on every SM (slower alone); whether that pays
+        # depends on the shape, so choose_attention_kernel() times both during warm-up unless the flag fixes it.
+        self.attn_share_sm = (ATTN_SHARE_SM == "on")
+        B.samkv_attn_share_sm(self.handle_attn, self.attn_share_sm)
         self.attn_stream = torch.cuda.Stream(device=device, priority=-1)
         self.groups = 8 if (w.n_layers % 8 == 0 and w.decode_steps == 0) else 1
         self.scores = torch.empty((L, Bt, Hkv, self.U_tot), dtype=torch.float32, device=device)
@@ -217,6 +225,28 @@ class Pipeline:
         for l in range(w.n_layers):
             kept += int((self.inv_map[l][:, :, self.tok_ids[l].long()] >= 0).sum())
         self.update_kept_rows = kept
+
+    def choose_attention_kernel(self, steps: int = 3):
+        """Warm-up time only: the overlapped schedule with either prefill attention kernel, the faster one stays."""
+        if ATTN_SHARE_SM != "auto" or self.groups <= 1:
+            return
+        best = None
+        for share in (False, True):
+            self.B.samkv_attn_share_sm(self.handle_attn, share)
+            for _ in range(2):
+                self.step()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(steps):
+                self.step()
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / steps
+            if best is None or ms < best[0]:
+                best = (ms, share)
+        self.attn_share_sm = best[1]
+        self.B.samkv_attn_share_sm(self.handle_attn, self.attn_share_sm)
 
     def sparsify(self):
         B, inp, w = self.B, self.inp, self.w
@@ -472,6 +502,7 @@ def e2e_steps(pipe: Pipeline, steps: int, warmup: int, host=None):
             O_host[l].copy_(pipe.O[l], non_blocking=True)
 
     O_ref = pipe.O.clone()                       # result of the device-resident steps: the e2e path must reproduce it
+    B.samkv_attn_share_sm(pipe.handle, pipe.attn_share_sm)      # (bit for bit: the same attention kernel as those steps)
     for _ in range(warmup):
         one_step()
     torch.cuda.synchronize()
@@ -486,6 +517,7 @@ def e2e_steps(pipe: Pipeline, steps: int, warmup: int, host=None):
     torch.cuda.synchronize()
     dev_s = e0.elapsed_time(e1) / 1e3
     wall_s = time.perf_counter() - t0
+    B.samkv_attn_share_sm(pipe.handle, False)
     return max(dev_s, wall_s) / steps, h2d, d2h
 
 
@@ -762,6 +794,7 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
     schedule where the workload has several layers, in order otherwise), then one in-order pass for the phases."""
     pipe = Pipeline(w, dev)
     pipe.prepare_recompute()
+    pipe.choose_attention_kernel()
     for _ in range(warmup):
         pipe.step()
     torch.cuda.synchronize()
@@ -797,6 +830,7 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
            "us_per_layer": ms * 1e3 / w.n_layers, "algorithmic_gb_per_step": ab["total"] / 1e9, "achieved_gbs": gbs,
            "frac_of_measured_copy_peak": gbs / hbm_peak, "frac_of_nominal_8tbs": gbs / HBM_NOMINAL_GBS,
            "schedule": "overlapped (8 layer groups)" if pipe.groups > 1 else "in order",
+           "attention_kernel_in_schedule": "leaves room on its SMs" if pipe.attn_share_sm else "default",
            "ms_per_step_scan_beside_attention": ms_scan,
            "in_order_phase_ms": phase, "in_order_ms_per_step": sum(phase.values()),
            "attention_tflops": attention_flops(w, pipe.S) / (phase["attn"] / 1e3) / 1e12 if phase.get("attn") else None,
@@ -822,11 +856,16 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling captures of a small case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling captures of a small case)")
     ap.add_argument("--budget-bp", type=int, default=0, help="override the sequence budget (basis points)")
+    ap.add_argument("--attn-share-sm", default="auto", choices=["auto", "on", "off"],
+                    help="prefill attention kernel of the overlapped schedule: the one that leaves room on its SMs "
+                         "(on), the default one (off), or whichever is faster during warm-up (auto)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the cfg4 budget sweep, cfg3 and the sustained loop that follow the timed region")
     args = ap.parse_args()
+    global ATTN_SHARE_SM
+    ATTN_SHARE_SM = args.attn_share_sm
     profiling_case = bool(args.layers or args.batch)       # small captures under a profiler: keep launches few
     if args.warmup < 3 and args.impl == "samkv" and not profiling_case:
         args.warmup = 3
@@ -861,6 +900,8 @@ def main():
 
     pipe = Pipeline(rank_workload(w, rank), dev)
     pipe.prepare_recompute()
+    if not profiling_case:                 # (small captures under a profiler keep the default kernel and few launches)
+        pipe.choose_attention_kernel()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()            # started early: nvidia-smi needs a moment before its first sample
@@ -967,6 +1008,8 @@ def main():
                      "frac_of_measured_copy_peak": pipeline_gbs / hbm_peak, "frac_of_nominal_8tbs": pipeline_gbs / HBM_NOMINAL_GBS,
                      "schedule": ("score+select, then %d layer groups: gather+update overlapped with attention on a second stream"
                                   % pipe.groups) if pipe.groups > 1 else "in order on one stream",
+                     "attention_kernel_in_schedule": ("128 rows, leaves room on its SMs (samkv_attn_share_sm)" if pipe.attn_share_sm
+                                                      else "default") + (", chosen during warm-up" if ATTN_SHARE_SM == "auto" else ""),
                      "timed_phase_ms": timed_phase_ms, "in_order_ms_per_step": sequential_ms,
                      "ms_per_step_scan_beside_attention": scan_ms,
                      "phase_ms": phase_ms, "other_calls_ms": widened, "sustained": sustained,

@@ -89,6 +89,13 @@ size_t samkv_workspace_bytes(const samkv_shape_t* shape, int32_t max_q_tokens, i
  * properties and enqueues one small memset on the default stream; allocates no device memory. */
 samkv_status_t samkv_create(samkv_handle_t* out, int device, void* workspace, size_t workspace_bytes);
 samkv_status_t samkv_destroy(samkv_handle_t h);
+/* Host-side switch of a handle (no GPU work, takes effect with the next samkv_attn call on the handle).
+ * on != 0: the caller keeps copy-like kernels (samkv_compact, samkv_update of other layers) running on another
+ * stream while attention is in flight.  samkv_attn then uses, for bf16 prefill chunks with d = 128 and at least
+ * 128 packed rows, a kernel that is slower on its own but leaves registers and shared memory on every SM for those
+ * kernels' CTAs; the default kernel fills its SMs.  Results obey the same bounds either way.  The paper has no
+ * counterpart: this is scheduling advice (Sec. 3.3 only fixes what attention computes). */
+samkv_status_t samkv_attn_share_sm(samkv_handle_t h, int32_t on);
 
 /* Synchronises `stream`, then returns SAMKV_ERR_DEVICE_CHECK if any kernel since the last poll
  * recorded a failed device-side check (and clears the record), SAMKV_ERR_CUDA if the stream

@@ -27,7 +27,7 @@ EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
            "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
            "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected",
-           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count", "samkv_select_compact",
+           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count", "samkv_attn_share_sm", "samkv_select_compact",
            "samkv_sparsify"]
 
 
@@ -94,6 +94,8 @@ def load_library(path: str) -> ctypes.CDLL:
     L.samkv_align.argtypes = [vp, shp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp]
     L.samkv_compact_protected.argtypes = [vp, shp, vp, vp, vp, vp, i32, vp, vp, vp]
     L.samkv_attn_kernel_count.argtypes = [vp, shp, i32, i32, i32]
+    L.samkv_attn_share_sm.argtypes = [vp, i32]
+    L.samkv_attn_share_sm.restype = i32
     L.samkv_attn_kernel_count.restype = i32
     L.samkv_block_means.argtypes = [vp, shp, vp, vp, vp]
     L.samkv_score_blocks.argtypes = L.samkv_score.argtypes
@@ -330,6 +332,10 @@ def samkv_score_blocks(handle: Handle, shape: Shape, Kbar, Q, T_q: int, Qloc, T_
                        qhat_out=None):
     _check(lib().samkv_score_blocks(handle.h, shape.ref(), _ptr(Kbar), _ptr(Q), T_q, _ptr(Qloc), T_loc, use_bias,
                                     _ptr(scores_out), _ptr(qhat_out), _stream()), "samkv_score_blocks")
+
+
+def samkv_attn_share_sm(handle: Handle, on: bool) -> None:
+    _check(lib().samkv_attn_share_sm(handle.h, int(bool(on))), "samkv_attn_share_sm")
 
 
 def samkv_attn_kernel_count(handle: Handle, shape: Shape, T_q: int, cache_capacity: int, appended: bool) -> int:

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsamkv.so")
 DEBUG_LIB_PATH = os.path.join(PKG_DIR, "libsamkv_debug.so")   # same sources with -DSAMKV_DEBUG_CHECKS (test hooks)
-SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "topp.cu", "align.cu", "means.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu", "attn_tc4.cu"]
+SOURCES = ["api.cu", "score.cu", "score_static.cu", "select.cu", "topp.cu", "align.cu", "means.cu", "compact.cu", "attn.cu", "attn_mma.cu", "attn_tc2.cu", "attn_tc3.cu", "attn_tc4.cu"]
 
 
 def nvcc_path() -> str:

@@ -175,6 +175,7 @@ samkv_status_t samkv_create(samkv_handle_t* out, int device, void* workspace, si
   h->workspace = static_cast<char*>(workspace);
   h->workspace_bytes = workspace_bytes;
   h->d_status = reinterpret_cast<int*>(workspace);
+  h->attn_share_sm = 0;
   if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
       cudaDeviceGetAttribute(&h->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess ||
       cudaMemsetAsync(workspace, 0, kStatusBytes, 0) != cudaSuccess) {
@@ -182,6 +183,14 @@ samkv_status_t samkv_create(samkv_handle_t* out, int device, void* workspace, si
     return SAMKV_ERR_CUDA;
   }
   *out = reinterpret_cast<samkv_handle_t>(h);
+  return SAMKV_OK;
+}
+
+samkv_status_t samkv_attn_share_sm(samkv_handle_t handle, int32_t on) {
+  samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
+  samkv_status_t st = check_handle(h);
+  if (st != SAMKV_OK) return st;
+  h->attn_share_sm = on ? 1 : 0;
   return SAMKV_OK;
 }
 
@@ -405,7 +414,7 @@ samkv_status_t samkv_attn(samkv_handle_t handle, const samkv_shape_t* shape, int
   if (!aligned16(Kc) || !aligned16(Vc) || !aligned16(Q) || !aligned16(O) || !aligned16(Kq) || !aligned16(Vq))
     return SAMKV_ERR_INVALID_ARG;
   if (Kq != nullptr && T_q > cache_capacity) return SAMKV_ERR_CAPACITY;
-  const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count);
+  const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count, h->attn_share_sm);
   const size_t ws_off = kStatusBytes + qhat_bytes(*shape);
   if (plan.partial_bytes > 0 && h->workspace_bytes < ws_off + plan.partial_bytes) return SAMKV_ERR_WORKSPACE;
   return from_cuda(launch_attn(*shape, layer, Kc, Vc, cache_capacity, cache_len, Q, T_q, Kq, Vq, scale, O, lse,
@@ -417,9 +426,9 @@ int32_t samkv_attn_kernel_count(samkv_handle_t handle, const samkv_shape_t* shap
   samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);
   Layout lo;
   if (h == nullptr || make_layout(shape, &lo) != SAMKV_OK || T_q < 1 || cache_capacity < 1) return 0;
-  const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count);
+  const AttnPlan plan = plan_attn(*shape, T_q, cache_capacity, h->sm_count, h->attn_share_sm);
   const bool self_merge = shape->dtype == SAMKV_BF16 && attn_merges_in_cluster(plan);
-  const bool self_append = shape->dtype == SAMKV_BF16 && shape->head_dim == 128 && plan.rows_per_cta == 128;
+  const bool self_append = shape->dtype == SAMKV_BF16 && shape->head_dim == 128 && plan.rows_per_cta == 128 && !plan.share_sm;
   int n = 1 + ((appended && !self_append) ? 1 : 0);
   if ((plan.n_splits > 1 || appended) && !self_merge) ++n;
   return n;

@@ -23,6 +23,9 @@ cudaError_t launch_attn_tc2(const samkv_shape_t& s, const void* Kc, const void* 
                             const int32_t* cache_len, const void* Q, int T_q, int appended, float scale, void* O,
                             float* lse, float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status,
                             cudaStream_t stream);
+cudaError_t launch_attn_tc3(const samkv_shape_t& s, const void* Kc, const void* Vc, int capacity, int32_t* cache_len,
+                            const void* Q, int T_q, int appended, float scale, void* O, float* lse, float* part_o,
+                            float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
 cudaError_t launch_attn_tc4(const samkv_shape_t& s, void* Kc, void* Vc, int capacity, int32_t* cache_len,
                             const void* Q, int T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
                             float* part_o, float2* part_ml, const AttnPlan& plan, int* d_status, cudaStream_t stream);
@@ -50,8 +53,9 @@ static long long best_split(long long base_ctas, long long tiles, long long slot
   return best_n;
 }
 
-AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) {
+AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count, int share_sm) {
   AttnPlan p;
+  p.share_sm = 0;
   const int G = s.n_q_heads / s.n_kv_heads;
   const int rows = T_q * G;
   const long long bh = (long long)s.batch * s.n_kv_heads;
@@ -72,6 +76,13 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count) 
     const bool use128 = cost128 <= cost256;
     p.rows_per_cta = use128 ? 128 : 256;
     p.n_splits = (int)(use128 ? n128 : n256);
+    if (share_sm && use128) {
+      // The caller runs copy kernels on other streams next to attention: the 128-row kernel with one double-buffered
+      // score tile (~2760 per tile + ~9000 per CTA) is slower alone but leaves them room on every SM.
+      long long cost_share = 0;
+      p.n_splits = (int)best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2760, 9000, &cost_share, 22000);
+      p.share_sm = 1;
+    }
   } else if (s.dtype == SAMKV_BF16) {
     // mma.sync kernel with 64 or 16 rows per CTA, 64-slot tiles; the fixed part is taken as 3 tiles
     p.rows_per_cta = rows > 16 ? 64 : 16;
@@ -322,7 +333,7 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   float2* part_ml = (float2*)(part_o + out_rows * plan.n_splits * kHeadDim);
 
   // the 128-row tensor-memory kernel writes the chunk's rows into the cache itself
-  const bool self_append = sizeof(T) == 2 && kHeadDim == 128 && plan.rows_per_cta == 128;
+  const bool self_append = sizeof(T) == 2 && kHeadDim == 128 && plan.rows_per_cta == 128 && !plan.share_sm;
   if (appended && !self_append) {
     const int row_bytes = kHeadDim * (int)sizeof(T);
     const long long threads = (long long)Bt * T_q * Hkv * (row_bytes / 16);
@@ -345,7 +356,10 @@ static cudaError_t launch_attn_t(const samkv_shape_t& s, int layer, void* Kc, vo
   const int G = Hq / Hkv;
   const int rows = T_q * G;
   if (sizeof(T) == 2) {
-    cudaError_t e = (plan.rows_per_cta == 128)
+    cudaError_t e = (plan.rows_per_cta == 128 && plan.share_sm)
+                        ? launch_attn_tc3(s, Kl, Vl, capacity, len_l, Q, T_q, appended, scale, O, lse, part_o, part_ml,
+                                          plan, d_status, stream)
+                    : (plan.rows_per_cta == 128)
                         ? launch_attn_tc4(s, Kl, Vl, capacity, len_l, Q, T_q, Kq, Vq, scale, O, lse, part_o, part_ml,
                                           plan, d_status, stream)
                     : (plan.rows_per_cta == 256)

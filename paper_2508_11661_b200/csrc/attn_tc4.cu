@@ -98,21 +98,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
-// Two non-negative finite fp32 values -> packed bf16 (lo in the low half), rounded to nearest with ties away from zero:
-// 0x8000 is added to the bit patterns and one byte permute takes the upper halves.  This keeps the conversion off the
-// special-function pipe, where cvt.rn.bf16x2.f32 runs at a quarter of the rate next to the exponentials.  (The
-// probabilities are <= 2^65 here, so the increment cannot carry into an infinity.)  lo and hi are replaced by the
-// rounded values: the row sum is taken over exactly what the tensor core multiplies with V, so that the rounding of
-// a dominant probability cancels between numerator and denominator instead of showing up in the output.
-__device__ __forceinline__ uint32_t round_pack_bf16(float& lo, float& hi) {
-  const uint32_t a = __float_as_uint(lo) + 0x8000u, b = __float_as_uint(hi) + 0x8000u;
-  uint32_t r;
-  asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(r) : "r"(a), "r"(b));
-  lo = __uint_as_float(a & 0xffff0000u);
-  hi = __uint_as_float(b & 0xffff0000u);
-  return r;
-}
-
 }  // namespace tc4
 
 // kPair: the grid is launched in clusters of two CTAs, the two KV splits of one (batch, kv head, query tile).  Each

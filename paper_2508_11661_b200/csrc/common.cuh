@@ -33,6 +33,7 @@ struct samkv_ctx_impl {
   char* workspace;
   size_t workspace_bytes;
   int* d_status;  // first word of the workspace
+  int attn_share_sm;  // samkv_attn_share_sm(): prefer the prefill attention kernel that leaves room on its SM
 };
 
 // ----- launchers implemented in the .cu files (all enqueue on `stream`, return cudaGetLastError) -------
@@ -74,8 +75,9 @@ struct AttnPlan {
   int n_splits;        // KV splits per (batch, kv head, row tile)
   int rows_per_cta;    // packed query rows (T_q * G) per CTA
   size_t partial_bytes;
+  int share_sm;        // 128 rows per CTA with the kernel that leaves registers and shared memory to other streams
 };
-AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count);
+AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count, int share_sm);
 // The 128-row tcgen05 kernel with exactly two KV splits merges them inside a two-CTA cluster: no merge kernel.
 inline bool attn_merges_in_cluster(const AttnPlan& p) { return p.rows_per_cta == 128 && p.n_splits == 2; }
 // Status block of the workspace (256 bytes, zero between calls): int 0 is the device check word, this int counts the

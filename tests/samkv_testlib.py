@@ -22,6 +22,9 @@ def oracle_k_units(w) -> list:
     return [O.budget_units(n, w.block_size, w.n_init, w.n_local, w.budget_bp) for n in w.ctx_lens]
 
 
+ATTN_SHARE_SM = False      # set by a fixture: every DeviceRun then asks for the SM-sharing attention kernel
+
+
 class DeviceRun:
     """One pass of the library over a workload; keeps every intermediate tensor."""
 
@@ -36,6 +39,8 @@ class DeviceRun:
         dev = inp["K"].device
         L, Bt, Hkv, d = w.n_layers, w.batch, w.n_kv_heads, w.head_dim
         self.handle = B.Handle(self.shape, max(w.q_tokens, 1), self.capacity)
+        if ATTN_SHARE_SM:                      # tests of the attention kernel that leaves room on its SM
+            B.samkv_attn_share_sm(self.handle, True)
         # outputs sit in front of canary words that no kernel may touch (checked by poll())
         self._guarded = []
 

@@ -153,7 +153,8 @@ def test_cfg4_stress_budget_sweep(budget_bp):
     _free_all()
 
 
-def test_cfg2_timed_schedule_matches_in_order_and_oracle():
+@pytest.mark.parametrize("share_sm", [False, True])
+def test_cfg2_timed_schedule_matches_in_order_and_oracle(share_sm):
     """The schedule bench.py times (scoring + selection of all layers, then 8 layer groups whose gather + update
     overlap the attention of earlier groups on a second stream, per-layer attention calls through a second handle)
     must give bit-identical results to the same calls issued in order on one stream, and its attention output
@@ -163,8 +164,13 @@ def test_cfg2_timed_schedule_matches_in_order_and_oracle():
     pipe = bench.Pipeline(w, torch.device(DEV))
     pipe.prepare_recompute()
     assert pipe.groups == 8 and pipe.R == 690
+    # either prefill attention kernel in the schedule; the in-order reference pass uses the same one
+    pipe.attn_share_sm = share_sm
+    B.samkv_attn_share_sm(pipe.handle_attn, share_sm)
+    B.samkv_attn_share_sm(pipe.handle, share_sm)
     pipe.step(overlap=False)
     torch.cuda.synchronize()
+    B.samkv_attn_share_sm(pipe.handle, False)
     ref = {"O": pipe.O.clone(), "sel": pipe.sel.clone(), "cache_len": pipe.cache_len.clone(),
            "Kc": pipe.Kc[::7].clone(), "Vc": pipe.Vc[::7].clone(), "scores": pipe.scores[::7].clone()}
     pipe.O.zero_(); pipe.sel.zero_(); pipe.cache_len.zero_(); pipe.Kc.zero_(); pipe.Vc.zero_(); pipe.scores.zero_()

@@ -526,6 +526,35 @@ def test_tensor_memory_attention_edge_shapes(ctx_lens, T_q, Hq, Hkv, budget_bp):
     full_check(w)
 
 
+@pytest.fixture
+def attention_shares_its_sm():
+    import samkv_testlib as T
+    T.ATTN_SHARE_SM = True
+    yield
+    T.ATTN_SHARE_SM = False
+
+
+SHARE_CASES = {
+    "cfg1": lambda: test_cfg1_llama_shape_bf16(),
+    "chunks": lambda: test_chunked_prefill_on_the_tensor_memory_kernel(),
+    "stream_order_on_q": lambda: test_attention_sees_q_written_by_the_kernel_right_before_it(),
+    "rows_160_many_splits": lambda: test_attention_row_tilings_and_long_cache(40, 4),
+    "rows_512_many_splits": lambda: test_attention_row_tilings_and_long_cache(64, 8),
+    "partial_tile": lambda: test_tensor_memory_attention_edge_shapes((40, 30), 32, 8, 2, 10000),
+    "single_row_tile": lambda: test_tensor_memory_attention_edge_shapes((100, 90), 129, 2, 2, 10000),
+    "g16": lambda: test_tensor_memory_attention_edge_shapes((200, 56), 16, 32, 2, 10000),
+    "g6_ragged": lambda: test_tensor_memory_attention_edge_shapes((700, 900, 333), 50, 12, 2, 3000),
+    "perturbation": lambda: test_a_five_percent_error_in_attention_would_be_caught(),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SHARE_CASES))
+def test_attention_kernel_that_leaves_room_on_its_sm(case, attention_shares_its_sm):
+    """samkv_attn_share_sm(handle, 1) routes bf16 prefill chunks to the double-buffered 128-row kernel (with the
+    separate append and merge launches where it needs them); the same cases and bounds as for the default kernel."""
+    SHARE_CASES[case]()
+
+
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_against_the_oracle(seed):
     """Seeded random small workloads: every stage of the path against the oracle (shapes no hand-written case covers)."""
