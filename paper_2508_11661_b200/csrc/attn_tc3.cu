@@ -322,14 +322,17 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
-          float p0 = fast_exp2(fmaf(sv[c0 + i], sl2, -mu));
-          float p1 = fast_exp2(fmaf(sv[c0 + i + 1], sl2, -mu));
-          float p2 = fast_exp2(fmaf(sv[c0 + i + 2], sl2, -mu));
-          float p3 = fast_exp2(fmaf(sv[c0 + i + 3], sl2, -mu));
-          // rounded first: the denominator sums exactly what the tensor core multiplies with V
-          pk[i >> 1] = round_pack_bf16(p0, p1);
-          pk[(i >> 1) + 1] = round_pack_bf16(p2, p3);
-          ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+          const float p0 = fast_exp2(fmaf(sv[c0 + i], sl2, -mu));
+          const float p1 = fast_exp2(fmaf(sv[c0 + i + 1], sl2, -mu));
+          const float p2 = fast_exp2(fmaf(sv[c0 + i + 2], sl2, -mu));
+          const float p3 = fast_exp2(fmaf(sv[c0 + i + 3], sl2, -mu));
+          // the denominator sums the rounded values, i.e. exactly what the tensor core multiplies with V (here the
+          // conversion instruction plus two integer operations per pair is cheaper than rounding on the integer pipe)
+          const uint32_t k01 = pack_bf16(p0, p1), k23 = pack_bf16(p2, p3);
+          pk[i >> 1] = k01;
+          pk[(i >> 1) + 1] = k23;
+          ps0 += __uint_as_float(k01 << 16); ps1 += __uint_as_float(k01 & 0xffff0000u);
+          ps2 += __uint_as_float(k23 << 16); ps3 += __uint_as_float(k23 & 0xffff0000u);
         }
         tmem_st16(tS + (c0 >> 1), pk);
       }
