@@ -99,6 +99,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
+  // Everything above needs nothing from the kernels before this one in the stream (they may still be running when
+  // this kernel was launched as a programmatic dependent); everything below does: Q, cache_len, the appended rows and
+  // the partial-result scratch.
+  pdl_wait();
+  int len = cache_len[b];     // (issued first: its latency overlaps the Q copies below)
+
   // Q tiles: cp.async by the softmax warps (rows beyond the chunk zero-filled); the MMA thread waits for Q_READY
   // before its first product
   if (warp < kSoftmaxWarps) {
@@ -113,11 +119,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
 
-  // Everything above needs nothing from the kernel before this one in the stream (it may still be running when this
-  // kernel was launched as its programmatic dependent); everything below does: cache_len, the appended rows and the
-  // partial-result scratch.
-  pdl_wait();
-  int len = cache_len[b];
   len = max(0, min(len, capacity));
   const int n_app = (appended && len + T_q <= capacity) ? T_q : 0;
   const int total = len + n_app;
