@@ -181,14 +181,16 @@ class Pipeline:
         # attention runs on its own high-priority stream with its own handle (own split-partial scratch), so
         # that the tensor-bound attention of one layer group overlaps the HBM-bound gather of the next
         self.shape1 = B.Shape.from_workload(w, n_layers=1)
-        self.handle_attn = B.Handle(self.shape1, w.q_tokens, self.capacity)
         # Its kernels run next to the gather and update of the following layers.  samkv_attn_share_sm asks for the
         # attention kernel that leaves registers and shared memory on every SM (slower alone); whether that pays
         # depends on the shape, so choose_attention_kernel() times both during warm-up unless the flag fixes it.
         self.attn_share_sm = (ATTN_SHARE_SM == "on")
-        B.samkv_attn_share_sm(self.handle_attn, self.attn_share_sm)
+        self.schedule_trials = {}
         self.attn_stream = torch.cuda.Stream(device=device, priority=-1)
-        self.groups = 8 if (w.n_layers % 8 == 0 and w.decode_steps == 0) else 1
+        # one attention call per group of layers (samkv_attn_layers); a handle per group count, because its workspace
+        # is sized for the group's requests
+        self._attn_handles = {}
+        self.set_groups(8 if (w.n_layers % 8 == 0 and w.decode_steps == 0) else 1)
         self.scores = torch.empty((L, Bt, Hkv, self.U_tot), dtype=torch.float32, device=device)
         self.sel = torch.empty((L, Bt, Hkv, sum(self.k_units)), dtype=torch.int32, device=device)
         self.Kc = torch.zeros((L, Bt, Hkv, self.capacity, d), dtype=w.torch_dtype, device=device)
@@ -226,27 +228,65 @@ class Pipeline:
             kept += int((self.inv_map[l][:, :, self.tok_ids[l].long()] >= 0).sum())
         self.update_kept_rows = kept
 
-    def choose_attention_kernel(self, steps: int = 3):
-        """Warm-up time only: the overlapped schedule with either prefill attention kernel, the faster one stays."""
-        if ATTN_SHARE_SM != "auto" or self.groups <= 1:
+    def attn_handle_for(self, groups: int):
+        B, w = self.B, self.w
+        if groups not in self._attn_handles:
+            wide = B.Shape.from_workload(w.replace(batch=w.batch * (w.n_layers // groups)), n_layers=1)
+            self._attn_handles[groups] = B.Handle(wide, w.q_tokens, self.capacity)
+        return self._attn_handles[groups]
+
+    def set_groups(self, groups: int):
+        """The schedule's layer groups: 1 = everything in order on one stream with one attention call for all layers;
+        g > 1 = gather + update of a group beside the attention of the previous groups."""
+        self.groups = groups
+        self.per_group = self.w.n_layers // groups
+        self.handle_attn = self.attn_handle_for(groups)
+        self.B.samkv_attn_share_sm(self.handle_attn, self.attn_share_sm if groups > 1 else False)
+
+    def choose_schedule(self, steps: int = 3):
+        """Warm-up time only: the step with 1, 2, 4 or 8 layer groups and, where groups overlap, with either prefill
+        attention kernel; the fastest combination stays.  --attn-share-sm on|off fixes the kernel."""
+        w = self.w
+        if w.n_layers % 8 != 0 or w.decode_steps > 0:
             return
+        shares = {"auto": (False, True), "on": (True,), "off": (False,)}[ATTN_SHARE_SM]
         best = None
-        for share in (False, True):
-            self.B.samkv_attn_share_sm(self.handle_attn, share)
-            for _ in range(2):
-                self.step()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(steps):
-                self.step()
-            b.record()
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / steps
-            if best is None or ms < best[0]:
-                best = (ms, share)
-        self.attn_share_sm = best[1]
-        self.B.samkv_attn_share_sm(self.handle_attn, self.attn_share_sm)
+        for groups in (1, 2, 4, 8):
+            for share in (shares if groups > 1 else (False,)):
+                self.attn_share_sm = share
+                self.set_groups(groups)
+                for _ in range(2):
+                    self.step()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(steps):
+                    self.step()
+                b.record()
+                torch.cuda.synchronize()
+                ms = a.elapsed_time(b) / steps
+                self.schedule_trials[f"{groups} groups" + (", sharing kernel" if share else "")] = ms
+                if best is None or ms < best[0]:
+                    best = (ms, groups, share)
+        self.attn_share_sm = best[2]
+        self.set_groups(best[1])
+
+    def attn_group(self, g: int):
+        """Attention of layer group g in one call (every layer's query chunk is available up front, as for the other
+        phases, which take all layers per call)."""
+        B, inp, w = self.B, self.inp, self.w
+        n = self.per_group
+        sl = slice(g * n, (g + 1) * n)
+        B.samkv_attn_layers(self.handle_attn, self.shape, g * n, n, self.Kc, self.Vc, self.capacity, self.cache_len,
+                            inp["Qa"][sl], w.q_tokens, inp["Kq"][sl], inp["Vq"][sl], 0.0, self.O[sl])
+
+    def attn_all(self):
+        """Attention of all layers in one call with the default kernel (the in-order phase table)."""
+        B, inp, w = self.B, self.inp, self.w
+        h = self.attn_handle_for(1)
+        B.samkv_attn_share_sm(h, False)
+        B.samkv_attn_layers(h, self.shape, 0, w.n_layers, self.Kc, self.Vc, self.capacity, self.cache_len, inp["Qa"],
+                            w.q_tokens, inp["Kq"], inp["Vq"], 0.0, self.O)
 
     def sparsify(self):
         B, inp, w = self.B, self.inp, self.w
@@ -255,7 +295,7 @@ class Pipeline:
         B.samkv_compact(self.handle, self.shape, inp["K"], inp["V"], self.sel, self.k_units, self.Kc, self.Vc,
                         self.capacity, self.cache_len, self.inv_map)
 
-    def step(self, ev=None, overlap=True):
+    def step(self, ev=None, overlap=True, attention_all_layers=False):
         """One pass of the whole path.  `ev` (optional) collects CUDA events at phase boundaries.
 
         overlap=True (the timed schedule): scoring and selection of all layers first; then, per group of layers,
@@ -294,10 +334,7 @@ class Pipeline:
                 ready.record(main)
                 with torch.cuda.stream(side):
                     side.wait_event(ready)
-                    for l in range(g * per, (g + 1) * per):
-                        B.samkv_attn(self.handle_attn, self.shape1, 0, self.Kc[l:l + 1], self.Vc[l:l + 1], self.capacity,
-                                     self.cache_len[l:l + 1], inp["Qa"][l], w.q_tokens, inp["Kq"][l], inp["Vq"][l], 0.0,
-                                     self.O[l])
+                    self.attn_group(g)
             main.wait_stream(side)
             mark("scan_overlapped_with_attn")
             return
@@ -323,10 +360,7 @@ class Pipeline:
                 ready.record(main)
                 with torch.cuda.stream(side):
                     side.wait_event(ready)
-                    for l in range(g * per, (g + 1) * per):
-                        B.samkv_attn(self.handle_attn, self.shape1, 0, self.Kc[l:l + 1], self.Vc[l:l + 1], self.capacity,
-                                     self.cache_len[l:l + 1], inp["Qa"][l], w.q_tokens, inp["Kq"][l], inp["Vq"][l], 0.0,
-                                     self.O[l])
+                    self.attn_group(g)
             main.wait_stream(side)
             mark("gather_update_attn_overlapped")
             return
@@ -337,9 +371,11 @@ class Pipeline:
             B.samkv_update(self.handle, self.shape, self.Kc, self.Vc, self.capacity, self.inv_map, self.tok_ids, self.R,
                            self.Knew, self.Vnew, B.SAMKV_UPDATE_FUSION)
         mark("update")
-        for l in range(w.n_layers):
-            B.samkv_attn(self.handle, self.shape, l, self.Kc, self.Vc, self.capacity, self.cache_len, inp["Qa"][l],
-                         w.q_tokens, inp["Kq"][l], inp["Vq"][l], 0.0, self.O[l])
+        if attention_all_layers and self.groups > 1:
+            self.attn_all()
+        else:
+            for g in range(self.groups):
+                self.attn_group(g)
         mark("attn")
         if w.decode_steps > 0:
             self.decode()
@@ -377,7 +413,8 @@ class Pipeline:
         # the timed schedule gathers and updates group by group
         n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + self.groups * per_group
         B = self.B
-        n += self.w.n_layers * B.samkv_attn_kernel_count(self.handle_attn, self.shape1, self.w.q_tokens, self.capacity, True)
+        wide = B.Shape.from_workload(self.w.replace(batch=self.w.batch * self.per_group), n_layers=1)
+        n += self.groups * B.samkv_attn_kernel_count(self.handle_attn, wide, self.w.q_tokens, self.capacity, True)
         return n + self.w.n_layers * self.w.decode_steps * B.samkv_attn_kernel_count(self.handle, self.shape, 1,
                                                                                     self.capacity, True)
 
@@ -497,12 +534,13 @@ def e2e_steps(pipe: Pipeline, steps: int, warmup: int, host=None):
             if pipe.R > 0:
                 B.samkv_update(pipe.handle, shape1, pipe.Kc[sl], pipe.Vc[sl], pipe.capacity, pipe.inv_map[sl],
                                pipe.tok_ids[sl], pipe.R, pipe.Knew[sl], pipe.Vnew[sl], B.SAMKV_UPDATE_FUSION)
-            B.samkv_attn(pipe.handle, shape1, 0, pipe.Kc[sl], pipe.Vc[sl], pipe.capacity, pipe.cache_len[sl],
-                         inp["Qa"][l], w.q_tokens, inp["Kq"][l], inp["Vq"][l], 0.0, pipe.O[l])
-            O_host[l].copy_(pipe.O[l], non_blocking=True)
+            if (l + 1) % pipe.per_group == 0:           # the group's caches are complete: its attention, as in the step
+                g = l // pipe.per_group
+                pipe.attn_group(g)
+                gs = slice(g * pipe.per_group, (g + 1) * pipe.per_group)
+                O_host[gs].copy_(pipe.O[gs], non_blocking=True)
 
     O_ref = pipe.O.clone()                       # result of the device-resident steps: the e2e path must reproduce it
-    B.samkv_attn_share_sm(pipe.handle, pipe.attn_share_sm)      # (bit for bit: the same attention kernel as those steps)
     for _ in range(warmup):
         one_step()
     torch.cuda.synchronize()
@@ -517,7 +555,6 @@ def e2e_steps(pipe: Pipeline, steps: int, warmup: int, host=None):
     torch.cuda.synchronize()
     dev_s = e0.elapsed_time(e1) / 1e3
     wall_s = time.perf_counter() - t0
-    B.samkv_attn_share_sm(pipe.handle, False)
     return max(dev_s, wall_s) / steps, h2d, d2h
 
 
@@ -794,7 +831,7 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
     schedule where the workload has several layers, in order otherwise), then one in-order pass for the phases."""
     pipe = Pipeline(w, dev)
     pipe.prepare_recompute()
-    pipe.choose_attention_kernel()
+    pipe.choose_schedule()
     for _ in range(warmup):
         pipe.step()
     torch.cuda.synchronize()
@@ -806,7 +843,10 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     ms_scan = None
-    if pipe.groups > 1:                                   # the other schedule: scan of the next group beside attention
+    chosen = (pipe.groups, pipe.attn_share_sm)
+    if w.n_layers % 8 == 0 and w.decode_steps == 0:       # the other schedule: scan of the next group beside attention
+        pipe.attn_share_sm = False
+        pipe.set_groups(8)
         for _ in range(warmup):
             pipe.step(overlap="scan")
         torch.cuda.synchronize()
@@ -816,21 +856,24 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
         e1.record()
         torch.cuda.synchronize()
         ms_scan = e0.elapsed_time(e1) / steps
+        pipe.attn_share_sm = chosen[1]
+        pipe.set_groups(chosen[0])
     phase = {}
     for _ in range(2):
         ev = []
-        pipe.step(ev, overlap=False)
+        pipe.step(ev, overlap=False, attention_all_layers=True)
         torch.cuda.synchronize()
         for (n0, a), (n1, b) in zip(ev[:-1], ev[1:]):
             phase[n1] = phase.get(n1, 0.0) + a.elapsed_time(b) / 2
-    status = max(pipe.B.samkv_poll_status(pipe.handle), pipe.B.samkv_poll_status(pipe.handle_attn))
+    status = max([pipe.B.samkv_poll_status(pipe.handle)] + [pipe.B.samkv_poll_status(h) for h in pipe._attn_handles.values()])
     ab = algorithmic_bytes(w, pipe.S, pipe.R, fusion=True, kept_rows=pipe.update_kept_rows)
     gbs = ab["total"] / (ms / 1e3) / 1e9
     out = {"layers_or_layer_buffers": w.n_layers, "budget_bp": w.budget_bp, "kept_tokens": pipe.S, "ms_per_step": ms,
            "us_per_layer": ms * 1e3 / w.n_layers, "algorithmic_gb_per_step": ab["total"] / 1e9, "achieved_gbs": gbs,
            "frac_of_measured_copy_peak": gbs / hbm_peak, "frac_of_nominal_8tbs": gbs / HBM_NOMINAL_GBS,
-           "schedule": "overlapped (8 layer groups)" if pipe.groups > 1 else "in order",
+           "schedule": ("overlapped (%d layer groups)" % pipe.groups) if pipe.groups > 1 else "in order",
            "attention_kernel_in_schedule": "leaves room on its SMs" if pipe.attn_share_sm else "default",
+           "schedule_trials_ms": pipe.schedule_trials or None,
            "ms_per_step_scan_beside_attention": ms_scan,
            "in_order_phase_ms": phase, "in_order_ms_per_step": sum(phase.values()),
            "attention_tflops": attention_flops(w, pipe.S) / (phase["attn"] / 1e3) / 1e12 if phase.get("attn") else None,
@@ -901,7 +944,7 @@ def main():
     pipe = Pipeline(rank_workload(w, rank), dev)
     pipe.prepare_recompute()
     if not profiling_case:                 # (small captures under a profiler keep the default kernel and few launches)
-        pipe.choose_attention_kernel()
+        pipe.choose_schedule()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()            # started early: nvidia-smi needs a moment before its first sample
@@ -929,7 +972,7 @@ def main():
     elapsed_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     elapsed_ms = max_over_ranks(elapsed_ms, dev)
-    status = max(pipe.B.samkv_poll_status(pipe.handle), pipe.B.samkv_poll_status(pipe.handle_attn))
+    status = max([pipe.B.samkv_poll_status(pipe.handle)] + [pipe.B.samkv_poll_status(h) for h in pipe._attn_handles.values()])
     if status != 0:
         raise RuntimeError(f"device-side check failed during the benchmark (status {status})")
 
@@ -944,11 +987,13 @@ def main():
     n_seq = 3
     for _ in range(n_seq):
         ev = []
-        pipe.step(ev, overlap=False)
+        pipe.step(ev, overlap=False, attention_all_layers=True)
         torch.cuda.synchronize()
         for (n0, a), (n1, b) in zip(ev[:-1], ev[1:]):
             phase_ms[n1] = phase_ms.get(n1, 0.0) + a.elapsed_time(b) / n_seq
     sequential_ms = sum(phase_ms.values())
+    if max(pipe.B.samkv_poll_status(h) for h in pipe._attn_handles.values()) != 0:
+        raise RuntimeError("device-side check failed in the in-order passes")
     phase_ms["score"] = timed_phase_ms["score"]          # the roofline figure comes from the timed steps
     widened = widened_rows_ms(pipe) if (rank == 0 and w.decode_steps == 0 and not profiling_case) else None
     # the same step looped for at least two seconds (board power and clocks settle; the headline region is short)
@@ -974,7 +1019,10 @@ def main():
 
     # the other schedule, outside the timed region: the whole scan of group g + 1 beside the attention of group g
     scan_ms = None
-    if rank == 0 and world == 1 and pipe.groups > 1 and not profiling_case:
+    if rank == 0 and world == 1 and w.n_layers % 8 == 0 and w.decode_steps == 0 and not profiling_case:
+        chosen = (pipe.groups, pipe.attn_share_sm)
+        pipe.attn_share_sm = False
+        pipe.set_groups(8)
         for _ in range(3):
             pipe.step(overlap="scan")
         torch.cuda.synchronize()
@@ -985,6 +1033,29 @@ def main():
         s1.record()
         torch.cuda.synchronize()
         scan_ms = s0.elapsed_time(s1) / 10
+        pipe.attn_share_sm = chosen[1]
+        pipe.set_groups(chosen[0])
+
+    # attention with one call per layer (what a caller that gets its queries layer by layer would run), for comparison
+    per_layer_attn_ms = None
+    if rank == 0 and world == 1 and w.decode_steps == 0 and not profiling_case:
+        def per_layer_calls():
+            pipe.cache_len.fill_(pipe.S)
+            for l in range(w.n_layers):
+                pipe.B.samkv_attn(pipe.handle, pipe.shape, l, pipe.Kc, pipe.Vc, pipe.capacity, pipe.cache_len, pipe.inp["Qa"][l],
+                                  w.q_tokens, pipe.inp["Kq"][l], pipe.inp["Vq"][l], 0.0, pipe.O[l])
+        for _ in range(2):
+            per_layer_calls()
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(5):
+            per_layer_calls()
+        s1.record()
+        torch.cuda.synchronize()
+        per_layer_attn_ms = s0.elapsed_time(s1) / 5
+        pipe.step()                                   # leave the caches and O as the timed schedule leaves them
+        torch.cuda.synchronize()
 
     ms_per_step = elapsed_ms / args.steps
     value = job_throughput(w, world, ms_per_step)
@@ -1007,11 +1078,16 @@ def main():
         "pipeline": {"algorithmic_gb_per_step": ab["total"] / 1e9, "achieved_gbs": pipeline_gbs,
                      "frac_of_measured_copy_peak": pipeline_gbs / hbm_peak, "frac_of_nominal_8tbs": pipeline_gbs / HBM_NOMINAL_GBS,
                      "schedule": ("score+select, then %d layer groups: gather+update overlapped with attention on a second stream"
-                                  % pipe.groups) if pipe.groups > 1 else "in order on one stream",
+                                  % pipe.groups) if pipe.groups > 1 else
+                                 ("in order on one stream, every phase one call over all layers" if w.decode_steps == 0 else "in order on one stream"),
                      "attention_kernel_in_schedule": ("128 rows, leaves room on its SMs (samkv_attn_share_sm)" if pipe.attn_share_sm
-                                                      else "default") + (", chosen during warm-up" if ATTN_SHARE_SM == "auto" else ""),
+                                                      else "default"),
+                     "schedule_trials_ms": pipe.schedule_trials or None,
                      "timed_phase_ms": timed_phase_ms, "in_order_ms_per_step": sequential_ms,
                      "ms_per_step_scan_beside_attention": scan_ms,
+                     "attention_ms_one_call_per_layer": per_layer_attn_ms,
+                     "attention_calls": "timed schedule: one samkv_attn_layers call per group of %d layers; in-order phase table: "
+                                        "one call for all layers, default kernel" % pipe.per_group,
                      "phase_ms": phase_ms, "other_calls_ms": widened, "sustained": sustained,
                      "attention_tflops_in_order": attention_flops(w, pipe.S) / (phase_ms["attn"] / 1e3) / 1e12 if phase_ms.get("attn") else None,
                      "bytes_note": "update charged for the rows it touches (new rows of every listed (token, head), old rows and "

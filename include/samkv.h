@@ -221,6 +221,19 @@ samkv_status_t samkv_attn(samkv_handle_t h, const samkv_shape_t* shape, int32_t 
                           int32_t cache_capacity, int32_t* cache_len, const void* Q, int32_t T_q, const void* Kq,
                           const void* Vq, float scale, void* O, float* lse, void* stream);
 
+/* The same attention for n consecutive layers, layer0 .. layer0 + n - 1, in one call: for callers that hold the
+ * queries of several layers at once (the data-parallel setting in which samkv_score .. samkv_update also take all
+ * layers per call).  One grid then covers every (layer, batch, KV head, row tile), which keeps all SMs busy where a
+ * single layer has fewer tiles than the GPU has SMs and leaves no gap between layers.
+ *   Kc, Vc, cache_len   as for samkv_attn (the whole [L, ...] tensors; the call offsets them to layer0)
+ *   Q, O                [n, Bt, T_q, Hq, d];  Kq, Vq [n, Bt, T_q, Hkv, d] optional;  lse [n, Bt, Hq, T_q] optional
+ * The workspace must be sized for the n * Bt requests of the call: samkv_workspace_bytes with a shape whose batch is
+ * n * Bt (SAMKV_ERR_WORKSPACE otherwise).  Per layer the result obeys the bounds of samkv_attn; the number of KV
+ * splits, and with it the rounding order, may differ from a per-layer call. */
+samkv_status_t samkv_attn_layers(samkv_handle_t h, const samkv_shape_t* shape, int32_t layer0, int32_t n, void* Kc,
+                                 void* Vc, int32_t cache_capacity, int32_t* cache_len, const void* Q, int32_t T_q,
+                                 const void* Kq, const void* Vq, float scale, void* O, float* lse, void* stream);
+
 /* ---- the paper's dynamic selection: Top-P per document, then Top-K across documents --------------- */
 
 #define SAMKV_MAX_STAR_LAYERS 64

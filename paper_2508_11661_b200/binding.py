@@ -27,7 +27,7 @@ EXPORTS = ["samkv_workspace_bytes", "samkv_create", "samkv_destroy", "samkv_poll
            "samkv_budget_units", "samkv_layout", "samkv_score", "samkv_select", "samkv_compact", "samkv_update",
            "samkv_attn", "samkv_score_static", "samkv_topp", "samkv_topp_plan", "samkv_select_cross",
            "samkv_select_cross_scratch_bytes", "samkv_compact_units", "samkv_align", "samkv_compact_protected",
-           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count", "samkv_attn_share_sm", "samkv_select_compact",
+           "samkv_block_means", "samkv_score_blocks", "samkv_attn_kernel_count", "samkv_attn_share_sm", "samkv_attn_layers", "samkv_select_compact",
            "samkv_sparsify"]
 
 
@@ -84,6 +84,8 @@ def load_library(path: str) -> ctypes.CDLL:
     L.samkv_select_compact.argtypes = [vp, shp, vp, i32p, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     L.samkv_sparsify.argtypes = [vp, shp, vp, vp, vp, i32, vp, i32, i32, i32p, vp, vp, vp, vp, i32, vp, vp, vp]
     L.samkv_attn.argtypes = [vp, shp, i32, vp, vp, i32, vp, vp, i32, vp, vp, f32, vp, vp, vp]
+    L.samkv_attn_layers.argtypes = [vp, shp, i32, i32, vp, vp, i32, vp, vp, i32, vp, vp, f32, vp, vp, vp]
+    L.samkv_attn_layers.restype = i32
     L.samkv_score_static.argtypes = [shp, vp, vp, i32, vp, i32, i32, vp, vp]
     f32p = ctypes.POINTER(ctypes.c_float)
     L.samkv_topp.argtypes = [vp, shp, vp, i32p, i32, vp, vp, vp, vp]
@@ -259,6 +261,15 @@ def samkv_attn(handle: Handle, shape: Shape, layer: int, Kc, Vc, cache_capacity:
     _check(lib().samkv_attn(handle.h, shape.ref(), layer, _ptr(Kc), _ptr(Vc), cache_capacity, _ptr(cache_len),
                             _ptr(Q), T_q, _ptr(Kq), _ptr(Vq), float(scale), _ptr(O), _ptr(lse), _stream()),
            "samkv_attn")
+
+
+def samkv_attn_layers(handle: Handle, shape: Shape, layer0: int, n: int, Kc, Vc, cache_capacity: int, cache_len, Q,
+                      T_q: int, Kq, Vq, scale: float, O, lse=None):
+    """n consecutive layers in one call; Q, O [n, Bt, T_q, Hq, d], Kq, Vq [n, Bt, T_q, Hkv, d].  The handle's
+    workspace must have been sized for n * Bt requests."""
+    _check(lib().samkv_attn_layers(handle.h, shape.ref(), layer0, n, _ptr(Kc), _ptr(Vc), cache_capacity,
+                                   _ptr(cache_len), _ptr(Q), T_q, _ptr(Kq), _ptr(Vq), float(scale), _ptr(O),
+                                   _ptr(lse), _stream()), "samkv_attn_layers")
 
 
 def samkv_score_static(shape: Shape, K, Q, T_q: int, Qloc, T_loc: int, use_bias: int, scores_out):

@@ -421,6 +421,24 @@ samkv_status_t samkv_attn(samkv_handle_t handle, const samkv_shape_t* shape, int
                                h->workspace + ws_off, plan, h->d_status, static_cast<cudaStream_t>(stream)));
 }
 
+samkv_status_t samkv_attn_layers(samkv_handle_t handle, const samkv_shape_t* shape, int32_t layer0, int32_t n,
+                                 void* Kc, void* Vc, int32_t cache_capacity, int32_t* cache_len, const void* Q,
+                                 int32_t T_q, const void* Kq, const void* Vq, float scale, void* O, float* lse,
+                                 void* stream) {
+  if (shape == nullptr || Kc == nullptr || Vc == nullptr || cache_len == nullptr) return SAMKV_ERR_INVALID_ARG;
+  if (layer0 < 0 || n < 1 || layer0 > shape->n_layers - n || cache_capacity < 1) return SAMKV_ERR_INVALID_ARG;
+  if ((long long)shape->batch * n > 0x7fffffffLL) return SAMKV_ERR_INVALID_ARG;
+  // Every tensor is contiguous over the layers, so n layers of Bt requests are one layer of n * Bt requests.
+  samkv_shape_t wide = *shape;
+  wide.n_layers = 1;
+  wide.batch = shape->batch * n;
+  const size_t elem = shape->dtype == SAMKV_BF16 ? 2 : 4;
+  const size_t layer_bytes = (size_t)shape->batch * shape->n_kv_heads * cache_capacity * shape->head_dim * elem;
+  return samkv_attn(handle, &wide, 0, static_cast<char*>(Kc) + layer0 * layer_bytes,
+                    static_cast<char*>(Vc) + layer0 * layer_bytes, cache_capacity,
+                    cache_len + (size_t)layer0 * shape->batch, Q, T_q, Kq, Vq, scale, O, lse, stream);
+}
+
 int32_t samkv_attn_kernel_count(samkv_handle_t handle, const samkv_shape_t* shape, int32_t T_q, int32_t cache_capacity,
                                 int32_t appended) {
   samkv_ctx_impl* h = reinterpret_cast<samkv_ctx_impl*>(handle);

@@ -530,6 +530,48 @@ def test_tensor_memory_attention_edge_shapes(ctx_lens, T_q, Hq, Hkv, budget_bp):
     full_check(w)
 
 
+@pytest.mark.parametrize("dtype,T_q,Hq,n,share", [("bf16", 64, 8, 3, False), ("bf16", 64, 8, 3, True), ("bf16", 32, 8, 2, False),
+                                                   ("bf16", 1, 8, 4, False), ("f32", 5, 4, 4, False)])
+def test_attention_of_several_layers_in_one_call(dtype, T_q, Hq, n, share):
+    """samkv_attn_layers over n of 4 layers (a range that starts at layer 1 where it can): every layer against the
+    oracle on its own cache, appended rows bit-exact in their layer's cache, cache lengths bumped for exactly the
+    layers of the call; tensor-memory kernels (both), the mma.sync kernel (decode row) and the fp32 kernel."""
+    w = synth.ragged_workload(ctx_lens=(700, 900, 333), dtype=dtype, head_dim=128 if dtype == "bf16" else 64,
+                              n_q_heads=Hq, n_kv_heads=2, q_tokens=T_q, n_init=4, n_local=8, budget_bp=3000,
+                              seed=99 + T_q).replace(n_layers=4, batch=2)
+    inp = {k: v.to(DEV) for k, v in synth.make_inputs(w, "cpu").items()}
+    run = DeviceRun(w, inp).sparsify()
+    torch.cuda.synchronize()
+    l0 = 4 - n if n < 4 else 0
+    handle = B.Handle(B.Shape.from_workload(w.replace(batch=w.batch * n), n_layers=1), T_q, run.capacity)
+    B.samkv_attn_share_sm(handle, share)
+    Kc0, Vc0 = run.Kc.clone(), run.Vc.clone()
+    sl = slice(l0, l0 + n)
+    Og = torch.empty_like(inp["Qa"][sl])
+    lse = torch.empty((n, w.batch, Hq, T_q), dtype=torch.float32, device=DEV)
+    B.samkv_attn_layers(handle, run.shape, l0, n, run.Kc, run.Vc, run.capacity, run.cache_len, inp["Qa"][sl], T_q,
+                        inp["Kq"][sl], inp["Vq"][sl], 0.0, Og, lse)
+    torch.cuda.synchronize()
+    assert B.samkv_poll_status(handle) == 0
+    for i, l in enumerate(range(l0, l0 + n)):
+        for b in range(w.batch):
+            err, K2, V2, m = check_attention(w, Kc0[l, b], Vc0[l, b], run.S, inp["Qa"][l, b], inp["Kq"][l, b],
+                                             inp["Vq"][l, b], Og[i, b], lse[i, b])
+            assert np.array_equal(to_f64(run.Kc[l, b][:, run.S:m]), K2[:, run.S:m])
+            assert np.array_equal(to_f64(run.Vc[l, b][:, run.S:m]), V2[:, run.S:m])
+    want = [[run.S + (T_q if l0 <= l < l0 + n else 0)] * w.batch for l in range(4)]
+    assert run.cache_len.cpu().tolist() == want
+    untouched = [l for l in range(4) if not (l0 <= l < l0 + n)]
+    for l in untouched:
+        assert torch.equal(run.Kc[l], Kc0[l]) and torch.equal(run.Vc[l], Vc0[l])
+    for bad_l0, bad_n in ((-1, 1), (0, 0), (3, 2), (0, 5)):                      # ranges outside the cache: refused
+        with pytest.raises(B.SamkvError) as e:
+            B.samkv_attn_layers(handle, run.shape, bad_l0, bad_n, run.Kc, run.Vc, run.capacity, run.cache_len,
+                                inp["Qa"][sl], T_q, None, None, 0.0, Og, None)
+        assert e.value.status == 1
+    assert run.poll() == 0
+
+
 @pytest.fixture
 def attention_shares_its_sm():
     import samkv_testlib as T
