@@ -186,6 +186,7 @@ class Pipeline:
         # depends on the shape, so choose_attention_kernel() times both during warm-up unless the flag fixes it.
         self.attn_share_sm = (ATTN_SHARE_SM == "on")
         self.schedule_trials = {}
+        self.fused_select = False
         self.attn_stream = torch.cuda.Stream(device=device, priority=-1)
         # one attention call per group of layers (samkv_attn_layers); a handle per group count, because its workspace
         # is sized for the group's requests
@@ -251,9 +252,10 @@ class Pipeline:
             return
         shares = {"auto": (False, True), "on": (True,), "off": (False,)}[ATTN_SHARE_SM]
         best = None
-        for groups in (1, 2, 4, 8):
+        for groups, fused in ((1, False), (1, True), (2, False), (4, False), (8, False)):
             for share in (shares if groups > 1 else (False,)):
                 self.attn_share_sm = share
+                self.fused_select = fused
                 self.set_groups(groups)
                 for _ in range(2):
                     self.step()
@@ -265,10 +267,12 @@ class Pipeline:
                 b.record()
                 torch.cuda.synchronize()
                 ms = a.elapsed_time(b) / steps
-                self.schedule_trials[f"{groups} groups" + (", sharing kernel" if share else "")] = ms
+                self.schedule_trials[f"{groups} groups" + (", sharing kernel" if share else "") +
+                                     (", fused select+compact" if fused else "")] = ms
                 if best is None or ms < best[0]:
-                    best = (ms, groups, share)
+                    best = (ms, groups, share, fused)
         self.attn_share_sm = best[2]
+        self.fused_select = best[3]
         self.set_groups(best[1])
 
     def attn_group(self, g: int):
@@ -295,7 +299,7 @@ class Pipeline:
         B.samkv_compact(self.handle, self.shape, inp["K"], inp["V"], self.sel, self.k_units, self.Kc, self.Vc,
                         self.capacity, self.cache_len, self.inv_map)
 
-    def step(self, ev=None, overlap=True, attention_all_layers=False):
+    def step(self, ev=None, overlap=True, attention_all_layers=False, fused_select=None):
         """One pass of the whole path.  `ev` (optional) collects CUDA events at phase boundaries.
 
         overlap=True (the timed schedule): scoring and selection of all layers first; then, per group of layers,
@@ -340,8 +344,10 @@ class Pipeline:
             return
         B.samkv_score(self.handle, self.shape, inp["K"], inp["Q"], w.q_tokens, inp["Qloc"], self.t_loc, 1, self.scores)
         mark("score")
-        B.samkv_select(self.handle, self.shape, self.scores, self.k_units, self.sel)
-        mark("select")
+        fused = (self.fused_select if fused_select is None else fused_select) and not (overlap and self.groups > 1)
+        if not fused:
+            B.samkv_select(self.handle, self.shape, self.scores, self.k_units, self.sel)
+            mark("select")
         if overlap and self.groups > 1:
             per = w.n_layers // self.groups
             shape_g = B.Shape.from_workload(w, n_layers=per)
@@ -364,9 +370,14 @@ class Pipeline:
             main.wait_stream(side)
             mark("gather_update_attn_overlapped")
             return
-        B.samkv_compact(self.handle, self.shape, inp["K"], inp["V"], self.sel, self.k_units, self.Kc, self.Vc,
-                        self.capacity, self.cache_len, self.inv_map)
-        mark("compact")
+        if fused:       # selection and gather of a (slab, context) by one CTA: no second launch, unit list not re-read
+            B.samkv_select_compact(self.handle, self.shape, self.scores, self.k_units, inp["K"], inp["V"], self.sel,
+                                   self.Kc, self.Vc, self.capacity, self.cache_len, self.inv_map)
+            mark("select_compact")
+        else:
+            B.samkv_compact(self.handle, self.shape, inp["K"], inp["V"], self.sel, self.k_units, self.Kc, self.Vc,
+                            self.capacity, self.cache_len, self.inv_map)
+            mark("compact")
         if self.R > 0:
             B.samkv_update(self.handle, self.shape, self.Kc, self.Vc, self.capacity, self.inv_map, self.tok_ids, self.R,
                            self.Knew, self.Vnew, B.SAMKV_UPDATE_FUSION)
@@ -412,6 +423,8 @@ class Pipeline:
             per_group += KERNELS_PER_CALL["update"]
         # the timed schedule gathers and updates group by group
         n = KERNELS_PER_CALL["score"] + KERNELS_PER_CALL["select"] + self.groups * per_group
+        if self.fused_select and self.groups == 1:
+            n -= 1                                       # selection and gather are one kernel
         B = self.B
         wide = B.Shape.from_workload(self.w.replace(batch=self.w.batch * self.per_group), n_layers=1)
         n += self.groups * B.samkv_attn_kernel_count(self.handle_attn, wide, self.w.q_tokens, self.capacity, True)
@@ -861,7 +874,7 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
     phase = {}
     for _ in range(2):
         ev = []
-        pipe.step(ev, overlap=False, attention_all_layers=True)
+        pipe.step(ev, overlap=False, attention_all_layers=True, fused_select=False)
         torch.cuda.synchronize()
         for (n0, a), (n1, b) in zip(ev[:-1], ev[1:]):
             phase[n1] = phase.get(n1, 0.0) + a.elapsed_time(b) / 2
@@ -987,7 +1000,7 @@ def main():
     n_seq = 3
     for _ in range(n_seq):
         ev = []
-        pipe.step(ev, overlap=False, attention_all_layers=True)
+        pipe.step(ev, overlap=False, attention_all_layers=True, fused_select=False)
         torch.cuda.synchronize()
         for (n0, a), (n1, b) in zip(ev[:-1], ev[1:]):
             phase_ms[n1] = phase_ms.get(n1, 0.0) + a.elapsed_time(b) / n_seq
@@ -1079,7 +1092,9 @@ def main():
                      "frac_of_measured_copy_peak": pipeline_gbs / hbm_peak, "frac_of_nominal_8tbs": pipeline_gbs / HBM_NOMINAL_GBS,
                      "schedule": ("score+select, then %d layer groups: gather+update overlapped with attention on a second stream"
                                   % pipe.groups) if pipe.groups > 1 else
-                                 ("in order on one stream, every phase one call over all layers" if w.decode_steps == 0 else "in order on one stream"),
+                                 (("in order on one stream, every phase one call over all layers" +
+                                   (", selection and gather fused (samkv_select_compact)" if pipe.fused_select else ""))
+                                  if w.decode_steps == 0 else "in order on one stream"),
                      "attention_kernel_in_schedule": ("128 rows, leaves room on its SMs (samkv_attn_share_sm)" if pipe.attn_share_sm
                                                       else "default"),
                      "schedule_trials_ms": pipe.schedule_trials or None,
