@@ -153,8 +153,8 @@ def test_cfg4_stress_budget_sweep(budget_bp):
     _free_all()
 
 
-@pytest.mark.parametrize("share_sm", [False, True])
-def test_cfg2_timed_schedule_matches_in_order_and_oracle(share_sm):
+@pytest.mark.parametrize("schedule", ["8 groups", "8 groups, sharing kernel", "in order, fused select+compact"])
+def test_cfg2_timed_schedule_matches_in_order_and_oracle(schedule):
     """The schedule bench.py times (scoring + selection of all layers, then 8 layer groups whose gather + update
     overlap the attention of earlier groups on a second stream, per-layer attention calls through a second handle)
     must give bit-identical results to the same calls issued in order on one stream, and its attention output
@@ -164,11 +164,17 @@ def test_cfg2_timed_schedule_matches_in_order_and_oracle(share_sm):
     pipe = bench.Pipeline(w, torch.device(DEV))
     pipe.prepare_recompute()
     assert pipe.groups == 8 and pipe.R == 690
-    # either prefill attention kernel in the schedule; the in-order reference pass uses the same one
+    # the schedules bench.py chooses from during warm-up; the reference pass issues separate calls in order on one
+    # stream, with the same attention calls (same layer grouping, same kernel) as the schedule under test
+    share_sm = schedule == "8 groups, sharing kernel"
     pipe.attn_share_sm = share_sm
-    B.samkv_attn_share_sm(pipe.handle_attn, share_sm)
+    if schedule.startswith("in order"):
+        pipe.set_groups(1)
+        pipe.fused_select = True
+    else:
+        B.samkv_attn_share_sm(pipe.handle_attn, share_sm)
     B.samkv_attn_share_sm(pipe.handle, share_sm)
-    pipe.step(overlap=False)
+    pipe.step(overlap=False, fused_select=False)
     torch.cuda.synchronize()
     B.samkv_attn_share_sm(pipe.handle, False)
     ref = {"O": pipe.O.clone(), "sel": pipe.sel.clone(), "cache_len": pipe.cache_len.clone(),
