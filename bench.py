@@ -915,6 +915,8 @@ def main():
     ap.add_argument("--attn-share-sm", default="auto", choices=["auto", "on", "off"],
                     help="prefill attention kernel of the overlapped schedule: the one that leaves room on its SMs "
                          "(on), the default one (off), or whichever is faster during warm-up (auto)")
+    ap.add_argument("--layer-groups", type=int, default=0, choices=[0, 1, 2, 4, 8],
+                    help="fix the number of layer groups of the schedule (1 = in order; 0 = choose during warm-up)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true",
@@ -956,7 +958,9 @@ def main():
 
     pipe = Pipeline(rank_workload(w, rank), dev)
     pipe.prepare_recompute()
-    if not profiling_case:                 # (small captures under a profiler keep the default kernel and few launches)
+    if args.layer_groups and w.n_layers % args.layer_groups == 0 and w.decode_steps == 0:
+        pipe.set_groups(args.layer_groups)
+    elif not profiling_case:               # (small captures under a profiler keep the default kernel and few launches)
         pipe.choose_schedule()
     sampler = ClockSampler(local_rank)
     if rank == 0:

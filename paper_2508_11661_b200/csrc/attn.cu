@@ -39,13 +39,14 @@ cudaError_t launch_attn_tc4(const samkv_shape_t& s, void* Kc, void* Vc, int capa
 // wave costs a whole wave.
 static long long best_split(long long base_ctas, long long tiles, long long slots, long long max_splits,
                             long long tile_cost, long long fixed_cost, long long* cost_out,
-                            long long fixed_cost_3plus = -1) {
+                            long long fixed_cost_3plus = -1, long long fixed_cost_2 = -1) {
   long long best_n = 1, best_cost = -1;
   for (long long n = 1; n <= max_splits; ++n) {
     const long long tps = (tiles + n - 1) / n;
     const long long waves = (base_ctas * n + slots - 1) / slots;
     // (a kernel that merges one or two splits itself pays more once partial results go through global memory)
-    const long long fixed = (n >= 3 && fixed_cost_3plus >= 0) ? fixed_cost_3plus : fixed_cost;
+    const long long fixed = (n >= 3 && fixed_cost_3plus >= 0) ? fixed_cost_3plus
+                            : (n == 2 && fixed_cost_2 >= 0)     ? fixed_cost_2 : fixed_cost;
     const long long cost = waves * (tps * tile_cost + fixed);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_n = n; }
   }
@@ -67,12 +68,14 @@ AttnPlan plan_attn(const samkv_shape_t& s, int T_q, int capacity, int sm_count, 
   if (s.dtype == SAMKV_BF16 && rows >= 128 && s.head_dim == 128) {
     // The two tcgen05 kernels, one CTA per SM, 128-slot tiles.  Measured on B200 (cycles): 256 rows per CTA
     // (two query tiles share every K/V tile, which halves the L2 traffic) ~4070 per tile + ~35000 per CTA;
-    // 128 rows per CTA (two groups of tiles taking turns) ~2150 per tile + ~8000 per CTA (~22000 with three or more splits, which go through global memory).  The second wins
-    // everywhere except on very long KV ranges.
+    // 128 rows per CTA (two groups of tiles taking turns) ~2150 per tile + ~8000 per CTA, ~25000 when two splits
+    // merge inside a cluster (the exchange, the partner's imbalance, and clusters that wait for two free SMs once the
+    // grid spans several waves), ~30000 with three or more splits, which go through global memory.  The second
+    // kernel wins everywhere except on very long KV ranges.
     const long long tiles = (capacity + 127) / 128;
     long long cost256 = 0, cost128 = 0;
     const long long n256 = best_split(bh * ((rows + 255) / 256), tiles, sm_count, max_splits, 4070, 35000, &cost256);
-    const long long n128 = best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2150, 8000, &cost128, 22000);
+    const long long n128 = best_split(bh * ((rows + 127) / 128), tiles, sm_count, max_splits, 2150, 8000, &cost128, 30000, 25000);
     const bool use128 = cost128 <= cost256;
     p.rows_per_cta = use128 ? 128 : 256;
     p.n_splits = (int)(use128 ? n128 : n256);
