@@ -801,6 +801,17 @@ def job_throughput(w, world: int, ms_per_step: float) -> float:
     return w.batch * w.l_tot * world / (ms_per_step / 1e3)
 
 
+def tensor_fractions(tflops: float) -> dict:
+    """Attention throughput (the two products, 4 * rows * slots * d flop) against the dense bf16 tensor peaks: the
+    measured cuBLAS figures of this machine (burst: a kernel timed alone; sustained: seconds under the power cap) and
+    the nominal 2250 TFLOP/s."""
+    peaks, kind = measured_peaks()
+    burst = float(peaks.get("bf16_tflops", 1590.0))
+    sustained = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    return {"of_measured_burst": tflops / burst, "of_measured_sustained": tflops / sustained, "of_nominal_2250": tflops / 2250.0,
+            "peak_kind": kind, "burst_tflops": burst, "sustained_tflops": sustained}
+
+
 def attention_flops(w, S: int) -> float:
     """QK^T and PV over the visible slots (cache + chunk; the causal part is counted in full), all layers."""
     return 4.0 * w.n_layers * w.batch * w.q_tokens * w.n_q_heads * (S + w.q_tokens) * w.head_dim
@@ -890,6 +901,7 @@ def run_other_workload(w, dev, hbm_peak: float, steps: int = 10, warmup: int = 3
            "ms_per_step_scan_beside_attention": ms_scan,
            "in_order_phase_ms": phase, "in_order_ms_per_step": sum(phase.values()),
            "attention_tflops": attention_flops(w, pipe.S) / (phase["attn"] / 1e3) / 1e12 if phase.get("attn") else None,
+           "attention_of_tensor_peak": tensor_fractions(attention_flops(w, pipe.S) / (phase["attn"] / 1e3) / 1e12) if phase.get("attn") else None,
            "device_status": status}
     if w.decode_steps > 0:
         out["decode"] = {"steps": w.decode_steps, "us_per_step": phase["decode"] * 1e3 / w.decode_steps / w.n_layers,
@@ -1109,6 +1121,7 @@ def main():
                                         "one call for all layers, default kernel" % pipe.per_group,
                      "phase_ms": phase_ms, "other_calls_ms": widened, "sustained": sustained,
                      "attention_tflops_in_order": attention_flops(w, pipe.S) / (phase_ms["attn"] / 1e3) / 1e12 if phase_ms.get("attn") else None,
+                     "attention_of_tensor_peak": tensor_fractions(attention_flops(w, pipe.S) / (phase_ms["attn"] / 1e3) / 1e12) if phase_ms.get("attn") else None,
                      "bytes_note": "update charged for the rows it touches (new rows of every listed (token, head), old rows and "
                                    "results only where the head kept the token); the inverse map and index lists are not charged",
                      "phase_gbs": {k: ab[k] / (phase_ms[k] / 1e3) / 1e9 for k in ("score", "compact", "update", "attn", "decode") if phase_ms.get(k, 0) > 0}},
