@@ -129,6 +129,12 @@ __device__ __forceinline__ uint4 fuse_vec(const uint4& nw, const uint4& od) {
   return ElemTraits<T>::pack(r);
 }
 
+// A CTA takes kUpdateRowsPerCta consecutive rows of one (layer, batch element).  The token -> slot look-ups
+// (tok_ids, then inv_map: two dependent trips to memory) are done once per row by one thread each and left in
+// shared memory; the copy loop then has a single trip per row (new and old rows are fetched together), two rows
+// per thread group in flight.
+constexpr int kUpdateRowsPerCta = 32;
+
 template <typename T, int kHeadDim>
 __global__ void __launch_bounds__(kCopyThreads)
 update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict__ inv_map,
@@ -136,52 +142,72 @@ update_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const int32_t* __restrict_
               int Hkv, int R, int L_tot, int capacity, int mode, long long n_rows, int* __restrict__ d_status) {
   constexpr int kPerVec = ElemTraits<T>::kPerVec;
   constexpr int kLanes = kHeadDim / kPerVec;
-  constexpr int kRowsPerCta = kCopyThreads / kLanes;
+  constexpr int kRowsPerPass = kCopyThreads / kLanes;
+  constexpr int kPasses = kUpdateRowsPerCta / kRowsPerPass;
+  static_assert(kPasses >= 2 && kPasses % 2 == 0 && kUpdateRowsPerCta <= kCopyThreads, "update tile shape");
   const int lane = threadIdx.x % kLanes;
+  const int group = threadIdx.x / kLanes;
   // blockIdx.y = l*Bt + b; blockIdx.x walks the R*Hkv rows of that (layer, batch element) in 32-bit arithmetic
   const int lb = blockIdx.y;
-  const int rh = blockIdx.x * kRowsPerCta + threadIdx.x / kLanes;                      // r*Hkv + h
-  const long long row = (long long)lb * (R * Hkv) + rh;                                // ((l*Bt + b)*R + r)*Hkv + h
+  const int rh0 = blockIdx.x * kUpdateRowsPerCta;                                      // first r*Hkv + h of the CTA
+  __shared__ int s_slot[kUpdateRowsPerCta];
+  if (threadIdx.x < kUpdateRowsPerCta) {
+    const int rh = rh0 + threadIdx.x;
+    const long long row = (long long)lb * (R * Hkv) + rh;                              // ((l*Bt + b)*R + r)*Hkv + h
+    int slot = -1;
+    if (rh < R * Hkv && row < n_rows) {
+      const int r = rh / Hkv, h = rh - r * Hkv;
+      const int l = lb / Bt;
+      const int t = tok_ids[(size_t)l * R + r];
+      const size_t slab = (size_t)lb * Hkv + h;
+      if (t >= 0 && t < L_tot) slot = inv_map[slab * L_tot + t];
+      // a token id past the sequence or a slot past the cache is skipped and reported (-1 is the regular "skip")
+      if (t >= L_tot || t < -1 || slot >= capacity) {
+        atomicMax(d_status, (int)CHECK_SEL_RANGE);
+        slot = -1;
+      }
+    }
+    s_slot[threadIdx.x] = slot;
+  }
+  __syncthreads();
   // Whole kLanes-groups take the same branch, and kLanes divides 32, so shuffles inside fuse_vec are
-  // executed by complete groups; inactive groups are masked out below without leaving the warp.
-  bool active = rh < R * Hkv && row < n_rows;
-  int slot = -1;
-  size_t slab = 0;
-  // the new rows depend on nothing but the row index: fetch them while the token -> slot look-ups are in flight
-  uint4 kn = make_uint4(0, 0, 0, 0), vn = kn, ko = kn, vo = kn;
-  if (active) {
-    const size_t src = (size_t)row * kHeadDim + lane * kPerVec;
-    kn = ld_stream(Knew + src);
-    vn = ld_stream(Vnew + src);
-  }
-  if (active) {
-    const int r = rh / Hkv, h = rh - r * Hkv;
-    const int l = lb / Bt;
-    const int t = tok_ids[(size_t)l * R + r];
-    slab = (size_t)lb * Hkv + h;
-    if (t >= 0 && t < L_tot) slot = inv_map[slab * L_tot + t];
-    // a token id past the sequence or a slot past the cache is skipped and reported (-1 is the regular "skip")
-    if (t >= L_tot || t < -1 || slot >= capacity) {
-      if (lane == 0) atomicMax(d_status, (int)CHECK_SEL_RANGE);
-      slot = -1;
+  // executed by complete groups; inactive groups are masked out without leaving the warp.
+#pragma unroll 1
+  for (int p = 0; p < kPasses; p += 2) {
+    uint4 kn[2], vn[2], ko[2], vo[2];
+    size_t dst[2];
+    bool active[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int i = (p + u) * kRowsPerPass + group;
+      const int rh = rh0 + i;
+      const int slot = s_slot[i];
+      active[u] = slot >= 0;
+      kn[u] = vn[u] = ko[u] = vo[u] = make_uint4(0, 0, 0, 0);
+      dst[u] = 0;
+      if (active[u]) {
+        const int h = rh % Hkv;
+        const size_t src = ((size_t)lb * (R * Hkv) + rh) * kHeadDim + lane * kPerVec;
+        dst[u] = (((size_t)lb * Hkv + h) * capacity + slot) * kHeadDim + lane * kPerVec;
+        kn[u] = ld_stream(Knew + src);
+        vn[u] = ld_stream(Vnew + src);
+        if (mode == SAMKV_UPDATE_FUSION) {
+          ko[u] = *reinterpret_cast<const uint4*>(Kc + dst[u]);
+          vo[u] = *reinterpret_cast<const uint4*>(Vc + dst[u]);
+        }
+      }
     }
-  }
-  active = slot >= 0;
-  size_t dst = 0;
-  if (active) {
-    dst = (slab * capacity + slot) * kHeadDim + lane * kPerVec;
-    if (mode == SAMKV_UPDATE_FUSION) {
-      ko = *reinterpret_cast<const uint4*>(Kc + dst);
-      vo = *reinterpret_cast<const uint4*>(Vc + dst);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (mode == SAMKV_UPDATE_FUSION) {
+        kn[u] = fuse_vec<T, kLanes>(kn[u], ko[u]);
+        vn[u] = fuse_vec<T, kLanes>(vn[u], vo[u]);
+      }
+      if (active[u]) {
+        *reinterpret_cast<uint4*>(Kc + dst[u]) = kn[u];
+        *reinterpret_cast<uint4*>(Vc + dst[u]) = vn[u];
+      }
     }
-  }
-  if (mode == SAMKV_UPDATE_FUSION) {
-    kn = fuse_vec<T, kLanes>(kn, ko);
-    vn = fuse_vec<T, kLanes>(vn, vo);
-  }
-  if (active) {
-    *reinterpret_cast<uint4*>(Kc + dst) = kn;
-    *reinterpret_cast<uint4*>(Vc + dst) = vn;
   }
 }
 
@@ -192,7 +218,7 @@ cudaError_t launch_update(const samkv_shape_t& s, int L_tot, void* Kc, void* Vc,
   if (n_rows == 0) return cudaSuccess;
 #define SAMKV_LAUNCH_UPDATE(T, HD)                                                                                 \
   do {                                                                                                             \
-    constexpr int rows_per_cta = kCopyThreads / (HD / ElemTraits<T>::kPerVec);                                     \
+    constexpr int rows_per_cta = kUpdateRowsPerCta;                                                                \
     const long long per_lb = ((long long)R * s.n_kv_heads + rows_per_cta - 1) / rows_per_cta;                      \
     const long long n_lb = (long long)s.n_layers * s.batch;                                                        \
     if (per_lb > 0x7fffffffLL || n_lb > 65535) return cudaErrorInvalidConfiguration;                               \
