@@ -44,7 +44,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
 __device__ __forceinline__ void select_context(const float* __restrict__ scores, int32_t* __restrict__ sel,
                                                const CtxTable& ct, const SelTable& st, int c, size_t slab, int U_tot,
                                                int S_u, uint32_t* keys, uint32_t* hist, uint32_t* warp_tot,
-                                               uint32_t* s_bin, uint32_t* s_remaining) {
+                                               uint32_t* s_bin, uint32_t* s_remaining, int32_t* list_s = nullptr) {
   const int base = ct.unit_off[c];
   const int nb = ct.unit_off[c + 1] - base;
   const int p0 = st.n_init_units[c];          // middle units are [p0, p1)
@@ -54,12 +54,21 @@ __device__ __forceinline__ void select_context(const float* __restrict__ scores,
   const int k_mid = k - (nb - n_mid);
   int32_t* out = sel + slab * S_u + st.sel_off[c];
   const int tid = threadIdx.x;
+  // every list entry also goes to list_s (shared memory) when the caller gathers right after the selection
+  auto emit = [&](int j, int unit) {
+    out[j] = unit;
+    if (list_s != nullptr) list_s[j] = unit;
+  };
 
-  for (int i = tid; i < p0; i += kSelThreads) out[i] = base + i;
-  for (int i = p1 + tid; i < nb; i += kSelThreads) out[k - (nb - p1) + (i - p1)] = base + i;
-  if (k_mid <= 0) return;
+  // (the protected units are emitted last: list_s may share its memory with the histograms)
+  auto emit_protected = [&]() {
+    for (int i = tid; i < p0; i += kSelThreads) emit(i, base + i);
+    for (int i = p1 + tid; i < nb; i += kSelThreads) emit(k - (nb - p1) + (i - p1), base + i);
+  };
+  if (k_mid <= 0) { emit_protected(); return; }
   if (k_mid >= n_mid) {
-    for (int i = tid; i < n_mid; i += kSelThreads) out[p0 + i] = base + p0 + i;
+    for (int i = tid; i < n_mid; i += kSelThreads) emit(p0 + i, base + p0 + i);
+    emit_protected();
     return;
   }
 
@@ -125,13 +134,14 @@ __device__ __forceinline__ void select_context(const float* __restrict__ scores,
   for (int i = a; i < b; ++i) {
     const uint32_t key = keys[i];
     if (key > pivot) {
-      out[p0 + gt_before + min(eq_before, need_eq)] = base + p0 + i;
+      emit(p0 + gt_before + min(eq_before, need_eq), base + p0 + i);
       ++gt_before;
     } else if (key == pivot) {
-      if (eq_before < need_eq) out[p0 + gt_before + eq_before] = base + p0 + i;
+      if (eq_before < need_eq) emit(p0 + gt_before + eq_before, base + p0 + i);
       ++eq_before;
     }
   }
+  emit_protected();
 }
 
 __global__ void __launch_bounds__(kSelThreads)
@@ -164,14 +174,17 @@ select_compact_kernel(const float* __restrict__ scores, int32_t* __restrict__ se
   const int c = (int)(blockIdx.x % ct.n_ctx);
   const size_t slab = blockIdx.x / ct.n_ctx;
   if (c == 0 && threadIdx.x == 0 && (slab % Hkv) == 0) cache_len[slab / Hkv] = S;
-  select_context(scores, sel, ct, st, c, slab, U_tot, S_u, keys, hist, warp_tot, &s_bin, &s_remaining);
+  // The context's unit list also stays in shared memory for the gather, in the histograms' memory (dead once the
+  // pivot is known), when it fits there.
+  int32_t* list_s = (st.sel_off[c + 1] - st.sel_off[c]) <= 4 * 256 ? reinterpret_cast<int32_t*>(hist) : nullptr;
+  select_context(scores, sel, ct, st, c, slab, U_tot, S_u, keys, hist, warp_tot, &s_bin, &s_remaining, list_s);
   __syncthreads();                             // the CTA's own list entries are visible to all of its threads
 
   constexpr int kLanes = kRowBytes / 16;
   constexpr int kRowsPerPass = kSelThreads / kLanes;
-  constexpr int kUnroll = 2;
+  constexpr int kUnroll = 4;
   const int lane = threadIdx.x % kLanes, rsub = threadIdx.x / kLanes;
-  const int32_t* list = sel + slab * S_u + st.sel_off[c];
+  const int32_t* list = list_s != nullptr ? list_s : sel + slab * S_u + st.sel_off[c];
   const int slot0 = st.slot_off[c], n_slots = st.slot_off[c + 1] - slot0;
   for (int r0 = 0; r0 < n_slots; r0 += kRowsPerPass * kUnroll) {
     uint4 kv[kUnroll], vv[kUnroll];
