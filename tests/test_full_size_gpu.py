@@ -153,6 +153,34 @@ def test_cfg4_stress_budget_sweep(budget_bp):
     _free_all()
 
 
+def test_bench_schedule_choice_on_a_small_workload():
+    """bench.py's warm-up trial of schedules (1, 2, 4, 8 layer groups, both prefill kernels, fused selection+gather)
+    on an 8-layer workload: whatever it picks, a step gives the results of the separate calls in order."""
+    import bench
+    w = synth.CONFIGS["cfg1"].replace(name="cfg1_8layers", n_layers=8, batch=2, q_tokens=64, recompute_share_bp=1500)
+    pipe = bench.Pipeline(w, torch.device(DEV))
+    pipe.prepare_recompute()
+    pipe.choose_schedule(steps=2)
+    assert pipe.groups in (1, 2, 4, 8) and len(pipe.schedule_trials) == 8
+    pipe.step()
+    torch.cuda.synchronize()
+    got = {"sel": pipe.sel.clone(), "Kc": pipe.Kc.clone(), "Vc": pipe.Vc.clone(), "len": pipe.cache_len.clone(),
+           "O": pipe.O.clone()}
+    pipe.O.zero_(); pipe.sel.zero_(); pipe.Kc.zero_(); pipe.Vc.zero_(); pipe.cache_len.zero_()
+    pipe.step(overlap=False, fused_select=False)
+    torch.cuda.synchronize()
+    assert torch.equal(got["sel"], pipe.sel) and torch.equal(got["len"], pipe.cache_len)
+    assert torch.equal(got["Kc"].view(torch.int16), pipe.Kc.view(torch.int16))
+    assert torch.equal(got["Vc"].view(torch.int16), pipe.Vc.view(torch.int16))
+    assert torch.equal(got["O"].view(torch.int16), pipe.O.view(torch.int16))
+    assert B.samkv_poll_status(pipe.handle) == 0 and B.samkv_poll_status(pipe.handle_attn) == 0
+    for (l, b) in ((0, 0), (7, 1)):
+        check_attention(w, pipe.Kc[l, b], pipe.Vc[l, b], pipe.S, pipe.inp["Qa"][l, b], pipe.inp["Kq"][l, b],
+                        pipe.inp["Vq"][l, b], pipe.O[l, b])
+    del pipe, got
+    _free_all()
+
+
 @pytest.mark.parametrize("schedule", ["8 groups", "8 groups, sharing kernel", "in order, fused select+compact"])
 def test_cfg2_timed_schedule_matches_in_order_and_oracle(schedule):
     """The schedule bench.py times (scoring + selection of all layers, then 8 layer groups whose gather + update
